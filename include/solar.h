@@ -1,0 +1,153 @@
+/*
+ * solar.h -- C ABI of the B200 (sm_100a) SVD-Attention forward pass.
+ *
+ * The operation is the one defined in Section 4.1 of the SOLAR paper
+ * (arxiv 2603.02561): every user's history matrix H (N x d, the shared
+ * key-value matrix) is replaced by its rank-r truncated SVD (Eq. 9); the left
+ * factor U cancels (Eq. 10), and M candidate queries attend over the r
+ * "factor tokens" sigma_i v_i^T projected by W_K / W_V (Eq. 11, Eq. 12), with
+ * the softmax kept (over the r tokens).
+ *
+ * Conventions shared by every entry point
+ *   - All tensors are dense, row-major, batch-major; "dt" is the STORAGE type of
+ *     H, C, W_Q, W_K, W_V, O and US.  Arithmetic accumulates in fp32 (or wider).
+ *   - Every pointer is a DEVICE pointer owned by the caller, 16-byte aligned,
+ *     valid until the work queued on `stream` has finished.  The library
+ *     allocates nothing and keeps no state between calls.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL =
+ *     the legacy default stream) and never synchronise.
+ *   - Errors the host can see (bad sizes, NULL or misaligned pointers, a
+ *     workspace that is too small) are returned BEFORE anything is launched.
+ *     Conditions only the device can see (Jacobi sweeps exhausted, non-finite
+ *     input) are written to info[] and never trap; such a user's outputs are
+ *     NaN-filled.
+ *   - Supported: d in {32, 64, 128}; 1 <= r <= min(d, N, 64); N >= 1; M >= 0;
+ *     B >= 0 (B == 0 or M == 0 makes the call a no-op returning SOLAR_OK).
+ *     Anything else returns SOLAR_ERR_UNSUPPORTED or SOLAR_ERR_INVALID_ARG.
+ *   - Two calls that share a workspace must not overlap on the GPU.
+ */
+#ifndef SOLAR_H_
+#define SOLAR_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SOLAR_OK = 0,
+  SOLAR_ERR_INVALID_ARG = 1, /* negative size, NULL / misaligned pointer, r out of range */
+  SOLAR_ERR_UNSUPPORTED = 2, /* d not in {32,64,128}, r > 64, unknown dtype or flag     */
+  SOLAR_ERR_WORKSPACE = 3,   /* workspace NULL or smaller than solar_workspace_bytes()   */
+  SOLAR_ERR_CUDA = 4         /* a CUDA runtime call or a launch failed                  */
+} solar_status_t;
+
+typedef enum { SOLAR_F32 = 0, SOLAR_BF16 = 1 } solar_dtype_t;
+
+/* flags of solar_svd_attention_fwd */
+enum {
+  SOLAR_FLAG_NO_SOFTMAX = 1 /* "SVD-Attn without Softmax" (ablation row of Table 4):
+                               O = scale * Query * Key_r^T * Value_r */
+};
+
+/* bits of info[b] written by the factorization */
+enum {
+  SOLAR_INFO_NOT_CONVERGED = 1, /* sweep cap reached before every rotation became negligible */
+  SOLAR_INFO_NONFINITE = 2      /* H_b^T H_b contains NaN or Inf; s, V of this user are NaN  */
+};
+
+const char* solar_status_string(solar_status_t st);
+
+/* Bytes of scratch that either call below needs for these sizes (the larger of
+ * the two).  Pure host arithmetic; returns 0 for unsupported sizes. */
+size_t solar_workspace_bytes(int B, int M, int N, int d, int r, solar_dtype_t dt);
+
+/*
+ * Rank-r truncated SVD of every H_b (Eq. 9), without forming U.
+ *
+ *   H    [B,N,d] dt   (in)   history embeddings, the shared key-value matrix
+ *   S    [B,r]  f32   (out)  singular values, descending
+ *   V    [B,d,r] f32  (out)  right singular vectors; V[b,j,i] = component j of v_i.
+ *                            Sign convention: the largest-magnitude component of
+ *                            each v_i is positive (lowest index wins a tie).
+ *   US   [B,N,r] dt   (out)  U*Sigma = H*V, or NULL to skip it (Eq. 10 removes U
+ *                            from the forward pass; it is offered for callers
+ *                            that want the left factor)
+ *   info [B] int      (out)  SOLAR_INFO_* bits per user, or NULL
+ *
+ * Route: G_b = H_b^T H_b is accumulated in one streaming pass over H, then a
+ * parallel Jacobi eigensolver diagonalises the d x d matrix in shared memory;
+ * s_i = sqrt(lambda_i).  M is accepted for a uniform signature and ignored.
+ */
+solar_status_t solar_lowrank_factor(int B, int M, int N, int d, int r, solar_dtype_t dt,
+                                    const void* H, float* S, float* V, void* US, int* info,
+                                    void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * SVD-Attention over the factor tokens (Eq. 11, Eq. 12):
+ *   Query   = C W_Q                      [M,d]
+ *   Key_r   = (V Sigma)^T W_K            [r,d]
+ *   Value_r = (V Sigma)^T W_V            [r,d]
+ *   O       = softmax_rows(scale * Query Key_r^T) Value_r      [M,d]
+ *
+ *   C        [B,M,d] dt (in)   candidate embeddings
+ *   S, V               (in)    as written by solar_lowrank_factor
+ *   Wq,Wk,Wv [d,d] dt   (in)   shared by all users; y = x W
+ *   scale               (in)   multiplies the scores (the paper prints none; 1/sqrt(d) is usual)
+ *   flags               (in)   0 or SOLAR_FLAG_NO_SOFTMAX
+ *   O        [B,M,d] dt (out)
+ *
+ * The M x r score matrix lives in registers / tensor memory only.  N is accepted
+ * for a uniform signature and ignored.
+ */
+solar_status_t solar_svd_attention_fwd(int B, int M, int N, int d, int r, solar_dtype_t dt,
+                                       const void* C, const float* S, const float* V,
+                                       const void* Wq, const void* Wk, const void* Wv,
+                                       float scale, unsigned flags, void* O,
+                                       void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------- *
+ * Stage-level entry points.  The two calls above are exactly
+ *   solar_lowrank_factor    = solar_gram_partials ; solar_eig_from_partials [; solar_project_us]
+ *   solar_svd_attention_fwd = solar_attn_prepare  ; solar_attn_apply
+ * on the same workspace.  They exist so that each kernel can be timed and
+ * checked on its own; argument meaning and rules are those given above.
+ * ------------------------------------------------------------------------- */
+
+/* Number of row-slices each H_b is cut into by solar_gram_partials (>= 1). */
+int solar_gram_splits(int B, int N, int d, solar_dtype_t dt);
+
+/* Streaming pass over H: slice s of user b contributes the d x d partial Gram
+ *   P[b,s] = sum over the rows n of slice s of h_n h_n^T        (fp32)
+ * stored at ((float*)workspace)[(b*splits + s)*d*d ...], row-major.
+ * H_b^T H_b (the matrix whose eigenvectors are V of Eq. 9) is the sum over s. */
+solar_status_t solar_gram_partials(int B, int N, int d, solar_dtype_t dt, const void* H,
+                                   void* workspace, size_t workspace_bytes, void* stream);
+
+/* Sums the partial Grams in slice order and diagonalises; writes S, V, info. */
+solar_status_t solar_eig_from_partials(int B, int N, int d, int r, solar_dtype_t dt,
+                                       float* S, float* V, int* info,
+                                       void* workspace, size_t workspace_bytes, void* stream);
+
+/* US = H V in the storage type (second pass over H). */
+solar_status_t solar_project_us(int B, int N, int d, int r, solar_dtype_t dt, const void* H,
+                                const float* V, void* US, void* stream);
+
+/* Per-user factor-token projections of Eq. 11 into the workspace:
+ * Value_r and the folded score operand T_b = scale * W_Q Key_r^T  (d x r). */
+solar_status_t solar_attn_prepare(int B, int d, int r, solar_dtype_t dt,
+                                  const float* S, const float* V,
+                                  const void* Wq, const void* Wk, const void* Wv, float scale,
+                                  void* workspace, size_t workspace_bytes, void* stream);
+
+/* Scores, softmax over the r tokens, weighted sum (Eq. 12), from the workspace
+ * written by solar_attn_prepare with the same B, d, r, dt. */
+solar_status_t solar_attn_apply(int B, int M, int d, int r, solar_dtype_t dt, const void* C,
+                                unsigned flags, void* O,
+                                void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SOLAR_H_ */

@@ -1,0 +1,169 @@
+// C ABI of the SVD-Attention forward pass: argument checks, workspace layout,
+// kernel selection.  Every host-visible error is returned before any launch.
+#include "solar_internal.cuh"
+
+using namespace solar;
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+solar_status_t check_dims(int B, int M, int N, int d, int r, solar_dtype_t dt) {
+  if (dt != SOLAR_F32 && dt != SOLAR_BF16) return SOLAR_ERR_UNSUPPORTED;
+  if (B < 0 || M < 0 || N < 1 || r < 1) return SOLAR_ERR_INVALID_ARG;
+  if (d != 32 && d != 64 && d != 128) return SOLAR_ERR_UNSUPPORTED;
+  if (r > d || r > N) return SOLAR_ERR_INVALID_ARG;
+  if (r > 64 || B > 65535) return SOLAR_ERR_UNSUPPORTED;
+  return SOLAR_OK;
+}
+
+solar_status_t check_ptr(const void* p) {
+  return (p != nullptr && aligned16(p)) ? SOLAR_OK : SOLAR_ERR_INVALID_ARG;
+}
+
+solar_status_t check_ws(const void* ws, size_t have, size_t need) {
+  if (ws == nullptr || !aligned16(ws) || have < need) return SOLAR_ERR_WORKSPACE;
+  return SOLAR_OK;
+}
+
+#define SOLAR_TRY(expr)                       \
+  do {                                        \
+    const solar_status_t st__ = (expr);       \
+    if (st__ != SOLAR_OK) return st__;        \
+  } while (0)
+
+solar_status_t from_cuda(cudaError_t e) { return e == cudaSuccess ? SOLAR_OK : SOLAR_ERR_CUDA; }
+
+}  // namespace
+
+extern "C" {
+
+const char* solar_status_string(solar_status_t st) {
+  switch (st) {
+    case SOLAR_OK: return "ok";
+    case SOLAR_ERR_INVALID_ARG: return "invalid argument";
+    case SOLAR_ERR_UNSUPPORTED: return "unsupported size, dtype or flag";
+    case SOLAR_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case SOLAR_ERR_CUDA: return "CUDA error";
+  }
+  return "unknown status";
+}
+
+size_t solar_workspace_bytes(int B, int M, int N, int d, int r, solar_dtype_t dt) {
+  if (check_dims(B, M, N, d, r, dt) != SOLAR_OK) return 0;
+  const size_t f = factor_ws_bytes(B, N, d), a = attn_ws_bytes(B, d, r);
+  const size_t need = f > a ? f : a;
+  return need ? need : 256;
+}
+
+int solar_gram_splits(int B, int N, int d, solar_dtype_t dt) {
+  if (check_dims(B, 0, N, d, 1, dt) != SOLAR_OK) return 0;
+  return gram_plan(B, N).splits;
+}
+
+solar_status_t solar_gram_partials(int B, int N, int d, solar_dtype_t dt, const void* H,
+                                   void* workspace, size_t workspace_bytes, void* stream) {
+  SOLAR_TRY(check_dims(B, 0, N, d, 1, dt));
+  if (B == 0) return SOLAR_OK;
+  SOLAR_TRY(check_ptr(H));
+  SOLAR_TRY(check_ws(workspace, workspace_bytes, factor_ws_bytes(B, N, d)));
+  const GramPlan plan = gram_plan(B, N);
+  return from_cuda(launch_gram_simt(B, N, d, dt, H, static_cast<float*>(workspace), plan,
+                                    static_cast<cudaStream_t>(stream)));
+}
+
+solar_status_t solar_eig_from_partials(int B, int N, int d, int r, solar_dtype_t dt, float* S,
+                                       float* V, int* info, void* workspace,
+                                       size_t workspace_bytes, void* stream) {
+  SOLAR_TRY(check_dims(B, 0, N, d, r, dt));
+  if (B == 0) return SOLAR_OK;
+  SOLAR_TRY(check_ptr(S));
+  SOLAR_TRY(check_ptr(V));
+  if (info != nullptr && (reinterpret_cast<uintptr_t>(info) & 3u)) return SOLAR_ERR_INVALID_ARG;
+  SOLAR_TRY(check_ws(workspace, workspace_bytes, factor_ws_bytes(B, N, d)));
+  const GramPlan plan = gram_plan(B, N);
+  return from_cuda(launch_eig_jacobi(B, d, r, static_cast<const float*>(workspace), plan.splits, S,
+                                     V, info, static_cast<cudaStream_t>(stream)));
+}
+
+solar_status_t solar_project_us(int B, int N, int d, int r, solar_dtype_t dt, const void* H,
+                                const float* V, void* US, void* stream) {
+  SOLAR_TRY(check_dims(B, 0, N, d, r, dt));
+  if (B == 0) return SOLAR_OK;
+  SOLAR_TRY(check_ptr(H));
+  SOLAR_TRY(check_ptr(V));
+  SOLAR_TRY(check_ptr(US));
+  return from_cuda(launch_project_us(B, N, d, r, dt, H, V, US, static_cast<cudaStream_t>(stream)));
+}
+
+solar_status_t solar_lowrank_factor(int B, int M, int N, int d, int r, solar_dtype_t dt,
+                                    const void* H, float* S, float* V, void* US, int* info,
+                                    void* workspace, size_t workspace_bytes, void* stream) {
+  (void)M;
+  SOLAR_TRY(check_dims(B, 0, N, d, r, dt));
+  if (B == 0) return SOLAR_OK;
+  SOLAR_TRY(check_ptr(H));
+  SOLAR_TRY(check_ptr(S));
+  SOLAR_TRY(check_ptr(V));
+  if (US != nullptr) SOLAR_TRY(check_ptr(US));
+  if (info != nullptr && (reinterpret_cast<uintptr_t>(info) & 3u)) return SOLAR_ERR_INVALID_ARG;
+  SOLAR_TRY(check_ws(workspace, workspace_bytes, factor_ws_bytes(B, N, d)));
+  SOLAR_TRY(solar_gram_partials(B, N, d, dt, H, workspace, workspace_bytes, stream));
+  SOLAR_TRY(solar_eig_from_partials(B, N, d, r, dt, S, V, info, workspace, workspace_bytes, stream));
+  if (US != nullptr) SOLAR_TRY(solar_project_us(B, N, d, r, dt, H, V, US, stream));
+  return SOLAR_OK;
+}
+
+solar_status_t solar_attn_prepare(int B, int d, int r, solar_dtype_t dt, const float* S,
+                                  const float* V, const void* Wq, const void* Wk, const void* Wv,
+                                  float scale, void* workspace, size_t workspace_bytes,
+                                  void* stream) {
+  SOLAR_TRY(check_dims(B, 0, r, d, r, dt));
+  if (B == 0) return SOLAR_OK;
+  SOLAR_TRY(check_ptr(S));
+  SOLAR_TRY(check_ptr(V));
+  SOLAR_TRY(check_ptr(Wq));
+  SOLAR_TRY(check_ptr(Wk));
+  SOLAR_TRY(check_ptr(Wv));
+  SOLAR_TRY(check_ws(workspace, workspace_bytes, attn_ws_bytes(B, d, r)));
+  return from_cuda(launch_attn_prepare(B, d, r, dt, S, V, Wq, Wk, Wv, scale,
+                                       static_cast<char*>(workspace), attn_ws_layout(d, r),
+                                       static_cast<cudaStream_t>(stream)));
+}
+
+solar_status_t solar_attn_apply(int B, int M, int d, int r, solar_dtype_t dt, const void* C,
+                                unsigned flags, void* O, void* workspace, size_t workspace_bytes,
+                                void* stream) {
+  SOLAR_TRY(check_dims(B, M, r, d, r, dt));
+  if (flags & ~(unsigned)SOLAR_FLAG_NO_SOFTMAX) return SOLAR_ERR_UNSUPPORTED;
+  if (B == 0 || M == 0) return SOLAR_OK;
+  SOLAR_TRY(check_ptr(C));
+  SOLAR_TRY(check_ptr(O));
+  SOLAR_TRY(check_ws(workspace, workspace_bytes, attn_ws_bytes(B, d, r)));
+  return from_cuda(launch_attn_simt(B, M, d, r, dt, C, flags, O, static_cast<const char*>(workspace),
+                                    attn_ws_layout(d, r), static_cast<cudaStream_t>(stream)));
+}
+
+solar_status_t solar_svd_attention_fwd(int B, int M, int N, int d, int r, solar_dtype_t dt,
+                                       const void* C, const float* S, const float* V,
+                                       const void* Wq, const void* Wk, const void* Wv, float scale,
+                                       unsigned flags, void* O, void* workspace,
+                                       size_t workspace_bytes, void* stream) {
+  (void)N;
+  SOLAR_TRY(check_dims(B, M, r, d, r, dt));
+  if (flags & ~(unsigned)SOLAR_FLAG_NO_SOFTMAX) return SOLAR_ERR_UNSUPPORTED;
+  if (B == 0 || M == 0) return SOLAR_OK;
+  SOLAR_TRY(check_ptr(C));
+  SOLAR_TRY(check_ptr(O));
+  SOLAR_TRY(check_ptr(S));
+  SOLAR_TRY(check_ptr(V));
+  SOLAR_TRY(check_ptr(Wq));
+  SOLAR_TRY(check_ptr(Wk));
+  SOLAR_TRY(check_ptr(Wv));
+  SOLAR_TRY(check_ws(workspace, workspace_bytes, attn_ws_bytes(B, d, r)));
+  SOLAR_TRY(solar_attn_prepare(B, d, r, dt, S, V, Wq, Wk, Wv, scale, workspace, workspace_bytes,
+                               stream));
+  return solar_attn_apply(B, M, d, r, dt, C, flags, O, workspace, workspace_bytes, stream);
+}
+
+}  // extern "C"

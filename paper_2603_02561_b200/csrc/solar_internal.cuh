@@ -1,0 +1,127 @@
+// Internal declarations shared by the kernels of the SVD-Attention forward pass.
+// Nothing here is part of the C ABI (include/solar.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "solar.h"
+
+namespace solar {
+
+constexpr int kNumSMs = 148;        // B200: 2 dies x 74 SMs
+constexpr int kGramTileRows = 128;  // rows of H per streamed tile
+constexpr int kMaxSplits = 64;
+constexpr int kMaxSweeps = 16;      // Jacobi sweep cap
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline size_t elem_size(solar_dtype_t dt) { return dt == SOLAR_BF16 ? 2 : 4; }
+
+// How each H_b is cut into row slices for the streaming Gram pass.  The cost
+// model is waves(B*S CTAs over the SMs) x (tiles per slice + fixed per-CTA cost).
+struct GramPlan {
+  int tiles;        // ceil(N / kGramTileRows)
+  int chunk_tiles;  // tiles per slice
+  int splits;       // slices per user (all non-empty)
+};
+
+inline GramPlan gram_plan(int B, int N) {
+  GramPlan p;
+  p.tiles = (N + kGramTileRows - 1) / kGramTileRows;
+  int best_s = 1;
+  long best_cost = -1;
+  const int smax = p.tiles < kMaxSplits ? p.tiles : kMaxSplits;
+  for (int s = 1; s <= smax; ++s) {
+    const int chunk = (p.tiles + s - 1) / s;
+    const int s_eff = (p.tiles + chunk - 1) / chunk;
+    const long waves = ((long)B * s_eff + kNumSMs - 1) / kNumSMs;
+    const long cost = waves * (chunk + 2);
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_s = s_eff; }
+  }
+  p.splits = best_s;
+  p.chunk_tiles = (p.tiles + best_s - 1) / best_s;
+  p.splits = (p.tiles + p.chunk_tiles - 1) / p.chunk_tiles;
+  return p;
+}
+
+// Workspace of the factorization: partial Grams [B][splits][d][d] fp32.
+inline size_t factor_ws_bytes(int B, int N, int d) {
+  const GramPlan p = gram_plan(B, N);
+  return align_up((size_t)B * p.splits * d * d * sizeof(float), 256);
+}
+
+// Workspace of the attention call, per user (all segments 256-byte aligned):
+//   Tf   [d][r] fp32   folded score operand  scale * W_Q Key_r^T
+//   Vr   [r][d] fp32   Value_r
+//   Thi  [r][d] bf16   high half of T^T  (tensor-core operand image)
+//   Tlo  [r][d] bf16   low half of T^T   (T^T - Thi)
+//   VrT  [d][r] bf16   Value_r^T         (tensor-core operand image)
+struct AttnWs {
+  size_t tf_off, vr_off, thi_off, tlo_off, vrt_off, per_user;
+};
+inline AttnWs attn_ws_layout(int d, int r) {
+  AttnWs w;
+  size_t o = 0;
+  w.tf_off = o;  o += align_up((size_t)d * r * 4, 256);
+  w.vr_off = o;  o += align_up((size_t)d * r * 4, 256);
+  w.thi_off = o; o += align_up((size_t)d * r * 2, 256);
+  w.tlo_off = o; o += align_up((size_t)d * r * 2, 256);
+  w.vrt_off = o; o += align_up((size_t)d * r * 2, 256);
+  w.per_user = o;
+  return w;
+}
+inline size_t attn_ws_bytes(int B, int d, int r) {
+  return attn_ws_layout(d, r).per_user * (size_t)B;
+}
+
+// ---- launchers (one per kernel file) --------------------------------------
+cudaError_t launch_gram_simt(int B, int N, int d, solar_dtype_t dt, const void* H, float* gpart,
+                             const GramPlan& plan, cudaStream_t st);
+cudaError_t launch_eig_jacobi(int B, int d, int r, const float* gpart, int splits, float* S,
+                              float* V, int* info, cudaStream_t st);
+cudaError_t launch_project_us(int B, int N, int d, int r, solar_dtype_t dt, const void* H,
+                              const float* V, void* US, cudaStream_t st);
+cudaError_t launch_attn_prepare(int B, int d, int r, solar_dtype_t dt, const float* S,
+                                const float* V, const void* Wq, const void* Wk, const void* Wv,
+                                float scale, char* ws, const AttnWs& lay, cudaStream_t st);
+cudaError_t launch_attn_simt(int B, int M, int d, int r, solar_dtype_t dt, const void* C,
+                             unsigned flags, void* O, const char* ws, const AttnWs& lay,
+                             cudaStream_t st);
+
+// ---- device helpers ----------------------------------------------------------
+template <typename T> __device__ __forceinline__ float to_f32(T x);
+template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) {
+  return __bfloat162float(x);
+}
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) {
+  return __float2bfloat16_rn(x);
+}
+
+// Loads 16 bytes of storage-type elements and widens them to fp32.
+template <typename T> struct Vec16;
+template <> struct Vec16<float> {
+  static constexpr int kElems = 4;
+  static __device__ __forceinline__ void load(const float* p, float* out) {
+    const float4 v = *reinterpret_cast<const float4*>(p);
+    out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+  }
+};
+template <> struct Vec16<__nv_bfloat16> {
+  static constexpr int kElems = 8;
+  static __device__ __forceinline__ void load(const __nv_bfloat16* p, float* out) {
+    const uint4 v = *reinterpret_cast<const uint4*>(p);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      out[2 * i] = __uint_as_float(w[i] << 16);
+      out[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+};
+
+}  // namespace solar

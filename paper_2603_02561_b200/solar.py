@@ -1,0 +1,188 @@
+"""ctypes binding of the C ABI in include/solar.h.
+
+Argument marshalling only: every step of the forward pass runs in the CUDA
+library.  torch is used for device memory and streams.  If the shared library
+is missing this module raises -- there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsolar_b200.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA = range(5)
+F32, BF16 = 0, 1
+FLAG_NO_SOFTMAX = 1
+INFO_NOT_CONVERGED, INFO_NONFINITE = 1, 2
+
+_c_int, _c_size, _c_vp, _c_float, _c_uint = (ctypes.c_int, ctypes.c_size_t, ctypes.c_void_p,
+                                              ctypes.c_float, ctypes.c_uint)
+
+# name -> (restype, argtypes); must list every symbol include/solar.h declares
+SIGNATURES = {
+    "solar_status_string": (ctypes.c_char_p, [_c_int]),
+    "solar_workspace_bytes": (_c_size, [_c_int] * 5 + [_c_int]),
+    "solar_lowrank_factor": (_c_int, [_c_int] * 5 + [_c_int] + [_c_vp] * 5 + [_c_vp, _c_size, _c_vp]),
+    "solar_svd_attention_fwd": (_c_int, [_c_int] * 5 + [_c_int] + [_c_vp] * 6 +
+                                [_c_float, _c_uint, _c_vp, _c_vp, _c_size, _c_vp]),
+    "solar_gram_splits": (_c_int, [_c_int] * 3 + [_c_int]),
+    "solar_gram_partials": (_c_int, [_c_int] * 3 + [_c_int, _c_vp, _c_vp, _c_size, _c_vp]),
+    "solar_eig_from_partials": (_c_int, [_c_int] * 4 + [_c_int] + [_c_vp] * 3 + [_c_vp, _c_size, _c_vp]),
+    "solar_project_us": (_c_int, [_c_int] * 4 + [_c_int] + [_c_vp] * 3 + [_c_vp]),
+    "solar_attn_prepare": (_c_int, [_c_int] * 3 + [_c_int] + [_c_vp] * 5 + [_c_float, _c_vp, _c_size, _c_vp]),
+    "solar_attn_apply": (_c_int, [_c_int] * 4 + [_c_int, _c_vp, _c_uint, _c_vp, _c_vp, _c_size, _c_vp]),
+}
+
+_lib = None
+
+
+class SolarError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().solar_status_string(status).decode()
+        super().__init__(f"{where}: {msg} (status {status})")
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libsolar_b200.so (built in-tree by build.py); raises if it is absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2603_02561_b200.build`; "
+                "this package has no CPU fallback")
+        L = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+def dtype_code(t: torch.dtype) -> int:
+    if t == torch.float32:
+        return F32
+    if t == torch.bfloat16:
+        return BF16
+    raise TypeError(f"storage dtype must be float32 or bfloat16, got {t}")
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise SolarError(status, where)
+
+
+def workspace_bytes(B, M, N, d, r, dtype) -> int:
+    return int(lib().solar_workspace_bytes(B, M, N, d, r, dtype_code(dtype)))
+
+
+def gram_splits(B, N, d, dtype) -> int:
+    return int(lib().solar_gram_splits(B, N, d, dtype_code(dtype)))
+
+
+def alloc_workspace(B, M, N, d, r, dtype, device="cuda") -> torch.Tensor:
+    return torch.empty(max(workspace_bytes(B, M, N, d, r, dtype), 256), dtype=torch.uint8, device=device)
+
+
+def _need(t, shape, dtype, name):
+    if t.dtype != dtype or tuple(t.shape) != tuple(shape) or not t.is_contiguous() or not t.is_cuda:
+        raise ValueError(f"{name}: want contiguous CUDA {dtype} {tuple(shape)}, got {t.dtype} {tuple(t.shape)}")
+
+
+def lowrank_factor(H, r, S=None, V=None, US=None, info=None, workspace=None, M=0, stream=None):
+    """solar_lowrank_factor: H[B,N,d] -> S[B,r], V[B,d,r] (and US[B,N,r] if given)."""
+    B, N, d = H.shape
+    _need(H, (B, N, d), H.dtype, "H")
+    dev = H.device
+    S = torch.empty(B, r, dtype=torch.float32, device=dev) if S is None else S
+    V = torch.empty(B, d, r, dtype=torch.float32, device=dev) if V is None else V
+    _need(S, (B, r), torch.float32, "S"); _need(V, (B, d, r), torch.float32, "V")
+    if US is not None:
+        _need(US, (B, N, r), H.dtype, "US")
+    if info is not None:
+        _need(info, (B,), torch.int32, "info")
+    if workspace is None:
+        workspace = alloc_workspace(B, M, N, d, r, H.dtype, dev)
+    st = lib().solar_lowrank_factor(B, M, N, d, r, dtype_code(H.dtype), _ptr(H), _ptr(S), _ptr(V),
+                                    _ptr(US), _ptr(info), _ptr(workspace), workspace.numel(),
+                                    _stream(stream))
+    _check(st, "solar_lowrank_factor")
+    return S, V
+
+
+def svd_attention_fwd(C, S, V, Wq, Wk, Wv, scale, flags=0, O=None, workspace=None, N=0, stream=None):
+    """solar_svd_attention_fwd: C[B,M,d] + factors -> O[B,M,d]."""
+    B, M, d = C.shape
+    r = S.shape[1]
+    _need(C, (B, M, d), C.dtype, "C")
+    _need(S, (B, r), torch.float32, "S"); _need(V, (B, d, r), torch.float32, "V")
+    for nm, W in (("Wq", Wq), ("Wk", Wk), ("Wv", Wv)):
+        _need(W, (d, d), C.dtype, nm)
+    O = torch.empty_like(C) if O is None else O
+    _need(O, (B, M, d), C.dtype, "O")
+    if workspace is None:
+        workspace = alloc_workspace(B, M, max(N, r), d, r, C.dtype, C.device)
+    st = lib().solar_svd_attention_fwd(B, M, max(N, r), d, r, dtype_code(C.dtype), _ptr(C), _ptr(S),
+                                       _ptr(V), _ptr(Wq), _ptr(Wk), _ptr(Wv), float(scale),
+                                       int(flags), _ptr(O), _ptr(workspace), workspace.numel(),
+                                       _stream(stream))
+    _check(st, "solar_svd_attention_fwd")
+    return O
+
+
+# ---- stage-level calls --------------------------------------------------------------
+def gram_partials(H, workspace, stream=None):
+    B, N, d = H.shape
+    _check(lib().solar_gram_partials(B, N, d, dtype_code(H.dtype), _ptr(H), _ptr(workspace),
+                                     workspace.numel(), _stream(stream)), "solar_gram_partials")
+
+
+def eig_from_partials(B, N, d, r, dtype, S, V, info, workspace, stream=None):
+    _check(lib().solar_eig_from_partials(B, N, d, r, dtype_code(dtype), _ptr(S), _ptr(V), _ptr(info),
+                                         _ptr(workspace), workspace.numel(), _stream(stream)),
+           "solar_eig_from_partials")
+
+
+def project_us(H, V, US, stream=None):
+    B, N, d = H.shape
+    r = V.shape[2]
+    _check(lib().solar_project_us(B, N, d, r, dtype_code(H.dtype), _ptr(H), _ptr(V), _ptr(US),
+                                  _stream(stream)), "solar_project_us")
+
+
+def attn_prepare(S, V, Wq, Wk, Wv, scale, workspace, stream=None):
+    B, d, r = V.shape
+    _check(lib().solar_attn_prepare(B, d, r, dtype_code(Wq.dtype), _ptr(S), _ptr(V), _ptr(Wq),
+                                    _ptr(Wk), _ptr(Wv), float(scale), _ptr(workspace),
+                                    workspace.numel(), _stream(stream)), "solar_attn_prepare")
+
+
+def attn_apply(C, r, flags, O, workspace, stream=None):
+    B, M, d = C.shape
+    _check(lib().solar_attn_apply(B, M, d, r, dtype_code(C.dtype), _ptr(C), int(flags), _ptr(O),
+                                  _ptr(workspace), workspace.numel(), _stream(stream)),
+           "solar_attn_apply")
+
+
+def forward(H, C, Wq, Wk, Wv, r, scale, flags=0, workspace=None, stream=None):
+    """The whole hot path: factorization then attention, back to back on one stream."""
+    B, N, d = H.shape
+    M = C.shape[1]
+    if workspace is None:
+        workspace = alloc_workspace(B, M, N, d, r, H.dtype, H.device)
+    S, V = lowrank_factor(H, r, workspace=workspace, M=M, stream=stream)
+    O = svd_attention_fwd(C, S, V, Wq, Wk, Wv, scale, flags, workspace=workspace, N=N, stream=stream)
+    return O, S, V
