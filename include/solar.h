@@ -147,6 +147,38 @@ solar_status_t solar_attn_apply(int B, int M, int d, int r, solar_dtype_t dt, co
                                 unsigned flags, void* O,
                                 void* workspace, size_t workspace_bytes, void* stream);
 
+/* ------------------------------------------------------------------------- *
+ * Factorization without caller-provided scratch.  (The paper has no counterpart:
+ * this is a packaging variant of solar_lowrank_factor, not another operation.)
+ *
+ * Some hosts of this library may not allocate device memory at all: a ranking
+ * server that carves every buffer out of an arena planned at start-up and
+ * forbids cudaMalloc while serving (it synchronises the device and can fail
+ * when the arena already fills the GPU), or a plug-in that is handed only its
+ * input and output tensors.  For them the partial-Gram scratch sits in a fixed
+ * 16 MiB array compiled into the library (solar_static_scratch_bytes()); every
+ * GPU that loads the library holds those 16 MiB until the process exits.
+ *
+ *   - Same arguments, outputs, info bits and rules as solar_lowrank_factor,
+ *     minus US and the workspace.  Calls no cudaMalloc / cudaFree and no
+ *     allocating library routine.
+ *   - Sizes whose scratch need, B * solar_gram_splits(B,N,d,dt) * d*d*4 bytes,
+ *     exceeds the array return SOLAR_ERR_WORKSPACE before anything is launched
+ *     (the headline shape B=16, N=10240, d=64 needs 2.25 MiB).
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current) and caches it; make that first call outside any
+ *     stream capture.
+ *   - All calls on a device share the one array: it keeps whatever the last call
+ *     left (every slice is fully overwritten before it is read, nothing needs
+ *     zeroing), and two calls that overlap on the GPU -- different streams,
+ *     or a call racing solar_eig_from_partials of another -- corrupt each other.
+ *     Serialise them on one stream or with events.
+ * ------------------------------------------------------------------------- */
+size_t solar_static_scratch_bytes(void);
+solar_status_t solar_lowrank_factor_static(int B, int M, int N, int d, int r, solar_dtype_t dt,
+                                           const void* H, float* S, float* V, int* info,
+                                           void* stream);
+
 #ifdef __cplusplus
 }
 #endif

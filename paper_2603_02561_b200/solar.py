@@ -34,6 +34,8 @@ SIGNATURES = {
     "solar_eig_from_partials": (_c_int, [_c_int] * 4 + [_c_int] + [_c_vp] * 3 + [_c_vp, _c_size, _c_vp]),
     "solar_project_us": (_c_int, [_c_int] * 4 + [_c_int] + [_c_vp] * 3 + [_c_vp]),
     "solar_attn_prepare": (_c_int, [_c_int] * 3 + [_c_int] + [_c_vp] * 5 + [_c_float, _c_vp, _c_size, _c_vp]),
+    "solar_static_scratch_bytes": (_c_size, []),
+    "solar_lowrank_factor_static": (_c_int, [_c_int] * 5 + [_c_int] + [_c_vp] * 4 + [_c_vp]),
     "solar_attn_apply": (_c_int, [_c_int] * 4 + [_c_int, _c_vp, _c_uint, _c_vp, _c_vp, _c_size, _c_vp]),
 }
 
@@ -141,6 +143,29 @@ def svd_attention_fwd(C, S, V, Wq, Wk, Wv, scale, flags=0, O=None, workspace=Non
                                        _stream(stream))
     _check(st, "solar_svd_attention_fwd")
     return O
+
+
+def static_scratch_bytes() -> int:
+    return int(lib().solar_static_scratch_bytes())
+
+
+def lowrank_factor_static(H, r, S=None, V=None, info=None, M=0, stream=None):
+    """solar_lowrank_factor_static: the factorization with the scratch inside the library.
+
+    For callers that cannot allocate device memory; takes only inputs and outputs.
+    Raises SolarError(ERR_WORKSPACE) when the sizes need more than static_scratch_bytes().
+    """
+    B, N, d = H.shape
+    _need(H, (B, N, d), H.dtype, "H")
+    if S is None or V is None:
+        raise ValueError("lowrank_factor_static allocates nothing: pass S[B,r] and V[B,d,r]")
+    _need(S, (B, r), torch.float32, "S"); _need(V, (B, d, r), torch.float32, "V")
+    if info is not None:
+        _need(info, (B,), torch.int32, "info")
+    st = lib().solar_lowrank_factor_static(B, M, N, d, r, dtype_code(H.dtype), _ptr(H), _ptr(S),
+                                           _ptr(V), _ptr(info), _stream(stream))
+    _check(st, "solar_lowrank_factor_static")
+    return S, V
 
 
 # ---- stage-level calls --------------------------------------------------------------
