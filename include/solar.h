@@ -54,8 +54,19 @@ enum {
 /* bits of info[b] written by the factorization */
 enum {
   SOLAR_INFO_NOT_CONVERGED = 1, /* sweep cap reached before every rotation became negligible */
-  SOLAR_INFO_NONFINITE = 2      /* H_b^T H_b contains NaN or Inf; s, V of this user are NaN  */
+  SOLAR_INFO_NONFINITE = 2,     /* H_b^T H_b contains NaN or Inf; s, V of this user are NaN  */
+  SOLAR_INFO_NOT_CERTIFIED = 4  /* only with SOLAR_ROUTE_SUBSPACE: the range-finder result was
+                                   written although its error bounds did not hold              */
 };
+
+/* How solar_eig_from_partials_ex reaches the top-r eigenpairs of H_b^T H_b.
+ * AUTO (what solar_lowrank_factor uses): Algorithm 1 (randomized range finder with
+ * power iteration) applied to the d x d Gram matrix, accepted per user only when
+ * residual and trace bounds certify the r pairs, else the full d x d Jacobi
+ * eigensolver.  SUBSPACE: the range finder alone, uncertified users flagged in
+ * info[].  FULL: the full eigensolver for every user (Eq. 9's exact truncated SVD
+ * whatever the spectrum). */
+enum { SOLAR_ROUTE_AUTO = 0, SOLAR_ROUTE_SUBSPACE = 1, SOLAR_ROUTE_FULL = 2 };
 
 const char* solar_status_string(solar_status_t st);
 
@@ -76,8 +87,10 @@ size_t solar_workspace_bytes(int B, int M, int N, int d, int r, solar_dtype_t dt
  *                            that want the left factor)
  *   info [B] int      (out)  SOLAR_INFO_* bits per user, or NULL
  *
- * Route: G_b = H_b^T H_b is accumulated in one streaming pass over H, then a
- * parallel Jacobi eigensolver diagonalises the d x d matrix in shared memory;
+ * Route: G_b = H_b^T H_b is accumulated in one streaming pass over H; its top-r
+ * eigenpairs come from Algorithm 1 (randomized range finder with power iteration)
+ * run on the d x d matrix in shared memory when its result can be certified, else
+ * from a parallel Jacobi eigensolver on the whole matrix (SOLAR_ROUTE_AUTO below);
  * s_i = sqrt(lambda_i).  M is accepted for a uniform signature and ignored.
  */
 solar_status_t solar_lowrank_factor(int B, int M, int N, int d, int r, solar_dtype_t dt,
@@ -129,6 +142,13 @@ solar_status_t solar_gram_partials(int B, int N, int d, solar_dtype_t dt, const 
 solar_status_t solar_eig_from_partials(int B, int N, int d, int r, solar_dtype_t dt,
                                        float* S, float* V, int* info,
                                        void* workspace, size_t workspace_bytes, void* stream);
+
+/* As above with the route chosen by the caller.  route_taken (device, [B] ints, or
+ * NULL) receives per user: route used (1 subspace, 2 full; 0 = non-finite input)
+ * | power steps << 8 | Jacobi sweeps << 16. */
+solar_status_t solar_eig_from_partials_ex(int B, int N, int d, int r, solar_dtype_t dt, int route,
+                                          float* S, float* V, int* info, int* route_taken,
+                                          void* workspace, size_t workspace_bytes, void* stream);
 
 /* US = H V in the storage type (second pass over H). */
 solar_status_t solar_project_us(int B, int N, int d, int r, solar_dtype_t dt, const void* H,

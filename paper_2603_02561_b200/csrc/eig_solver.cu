@@ -1,0 +1,779 @@
+// Batched symmetric eigensolver for the Gram matrices: G_b = V Lambda V^T, top-r
+// pairs only, one CTA per user, everything in shared memory.  The top-r
+// eigenpairs give the truncated SVD of Eq. 9 without U: s_i = sqrt(lambda_i).
+//
+// Two routes inside the one kernel:
+//
+//  (1) Subspace route -- Algorithm 1 (randomized range finder with power
+//      iteration) applied to the Gram matrix: Omega is Gaussian, each power step
+//      is Y = G Z followed by a Cholesky-QR in double precision, and the small
+//      SVD at the end of Algorithm 1 becomes the p x p Rayleigh-Ritz problem
+//      T = Z^T G Z, solved by parallel two-sided Jacobi (p = 8, 16 or 32 >= r).
+//      The result is accepted only if it is CERTIFIED a posteriori: the residuals
+//      G v_i - theta_i v_i must be small against the gaps of the Ritz values, and
+//      the trace of G must show that nothing outside the kept r pairs can reach
+//      theta_r.  Otherwise the CTA falls through to route (2).
+//
+//  (2) Full route -- parallel two-sided Jacobi on the whole d x d matrix, always
+//      valid (Eq. 9's exact truncated SVD for any spectrum).
+//
+// Jacobi rounds use the round-robin tournament ordering (n/2 disjoint pairs per
+// round, n-1 rounds per sweep).  In one round every 2x2 block
+// G[{p,q}][{p',q'}] is touched by exactly one thread, which applies the row
+// pair's rotation from the left and the column pair's from the right.  Each
+// thread recomputes the (at most four) rotations it needs from the diagonal
+// blocks of the current matrix, and the matrix is double-buffered, so a round
+// costs ONE barrier.
+#include <math.h>
+
+#include "solar_internal.cuh"
+
+namespace solar {
+
+namespace {
+
+constexpr float kTolRel = 2.3841858e-07f;  // 2^-22: |g_pq| <= tol*sqrt(g_pp g_qq) counts as zero
+constexpr float kTolAbs = 7.4505806e-09f;  // 2^-27 of the largest diagonal entry
+constexpr float kUnit = 5.9604645e-08f;    // 2^-24, fp32 unit roundoff
+constexpr int kMaxSubspaceIters = 3;       // power steps before the subspace route gives up
+
+// Acceptance thresholds of the subspace route (chosen by the storage type).
+struct EigTol {
+  float eps_vec;     // certified bound on sin(angle) of every kept vector
+  float floor_rel;   // residuals below floor_rel*theta_1 are at the rounding level of fp32
+  float sweep_stop;  // a Jacobi sweep whose largest relative off-diagonal was below this is the last
+};
+
+template <int D> struct EigCfg {
+  static constexpr int NP = D / 2;                 // pairs per round
+  static constexpr int PT = (D == 128) ? 2 : 1;    // row pairs (and column pairs) per thread
+  static constexpr int SIDE = NP / PT;             // threads along each side of the block grid
+  static constexpr int THREADS = SIDE * SIDE;
+  static constexpr int LD = D + 4;                 // rows stay 16-byte aligned
+  static constexpr int PMAX = (D >= 64) ? 32 : 16; // largest subspace dimension (<= D/2)
+  static constexpr int LP = PMAX + 1;
+  static constexpr int LPD = PMAX + 2;             // row pitch of the double matrices (16-byte rows)
+  // floats of the full route: Gc, Gn, Vm, lam[D], order[D]
+  static constexpr int FULL_FLOATS = 3 * D * LD + 2 * D;
+  // floats of the subspace route: Ad, Li [PMAX][LPD], dref [PMAX] (double, first: 16-byte aligned),
+  // Zb, Yb, Xb [D][PMAX], Tc, Tn, Wm [PMAX][LP], theta, res2, ordp [PMAX], pad
+  static constexpr int SUB_FLOATS = 2 * (2 * PMAX * LPD + PMAX) + 3 * D * PMAX + 3 * PMAX * LP +
+                                    3 * PMAX + 3;
+  // D = 128: the subspace buffers alias Gn and Vm (free until the full route starts)
+  static constexpr bool ALIAS = (D == 128);
+  static constexpr size_t SMEM =
+      (size_t)(FULL_FLOATS + (ALIAS ? 0 : SUB_FLOATS)) * sizeof(float);
+  static_assert(!ALIAS || SUB_FLOATS <= 2 * D * LD, "subspace buffers must fit in Gn+Vm");
+  static_assert((D * LD) % 4 == 0 && FULL_FLOATS % 4 == 0, "16-byte alignment of the regions");
+};
+
+// Rotation J = [[c, s], [-s, c]] that annihilates g_pq of the 2x2 symmetric block
+// [[a, g], [g, b]]; identity when g is negligible (or not a number).  Returned
+// as s, tau = s/(1+c) and t = s/c: columns are updated in the cancellation-free
+// form x_p' = x_p - s (x_q + tau x_p), x_q' = x_q + s (x_p - tau x_q), and the
+// diagonal as a' = a - t g, b' = b + t g, so a near-identity rotation perturbs
+// the matrix by O(s) instead of by a rounding error of the full entry.
+// `big` is set when the rotated pair had g^2 > stop2 |a b|.  The matrix is scaled so
+// that its largest diagonal entry lies in [1, 2): squares cannot overflow, and entries
+// whose squares underflow are below the absolute threshold.  The approximate rsqrt
+// (2 ulp) only moves the rotation angle by a rounding error.
+struct Rot { float s, tau, t; };
+
+__device__ __forceinline__ Rot jacobi_rot(float a, float b, float g, float thr_abs2, float stop2,
+                                          bool& big) {
+  const float g2 = g * g;
+  const float ab = fabsf(a * b);
+  const bool act = (g2 > thr_abs2) && (g2 > (kTolRel * kTolRel) * ab);
+  big = act && (g2 > stop2 * ab);
+  // With d = b - a and h = sqrt(d^2 + 4 g^2):  cos^2 = (h + |d|) / (2 h),
+  // sin = sgn(d) g / (h cos),  tan = sin / cos,  tau = sin / (1 + cos).
+  // Two dependent special-function evaluations (both rsqrt); 1 / (1 + cos), with
+  // 1 + cos in [1.707, 2], comes from a linear guess and two Newton steps.
+  const float dlt = b - a;
+  const float rh = rsqrtf(fmaf(dlt, dlt, 4.f * g2));
+  const float c2 = fmaf(0.5f * fabsf(dlt), rh, 0.5f);
+  const float rc = rsqrtf(c2);
+  const float c = c2 * rc;
+  const float s = copysignf(g * rh, dlt * g) * rc;
+  const float t = s * rc;
+  const float u = 1.f + c;
+  float y = fmaf(-0.29289f, u, 1.08579f);
+  y = y * fmaf(-u, y, 2.f);
+  y = y * fmaf(-u, y, 2.f);
+  Rot r;
+  r.s = act ? s : 0.f;
+  r.t = act ? t : 0.f;
+  r.tau = act ? s * y : 0.f;
+  return r;
+}
+
+// Players (a, c) of pair i in the circle method on n players, advanced by one round:
+// pair 0 is (n-1, k); pair i > 0 is (k+i, k-i) modulo n-1.
+__device__ __forceinline__ void pair_start(int i, int n, int& a, int& c) {
+  a = (i == 0) ? n - 1 : i;
+  c = (i == 0) ? 0 : n - 1 - i;
+}
+__device__ __forceinline__ void pair_next(int i, int n, int& a, int& c) {
+  const int up_a = (a + 1 == n - 1) ? 0 : a + 1;
+  a = (i == 0) ? a : up_a;
+  c = (c + 1 == n - 1) ? 0 : c + 1;
+}
+
+__device__ __forceinline__ void rot_apply(const Rot& r, float& xp, float& xq) {
+  const float p = xp, q = xq;
+  xp = fmaf(-r.s, fmaf(r.tau, p, q), p);
+  xq = fmaf(r.s, fmaf(-r.tau, q, p), q);
+}
+
+// Barrier among the first `nthreads` threads of the CTA (a multiple of 32).
+__device__ __forceinline__ void bar_named(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// Integer mixer (two multiply-xorshift rounds) used as a counter-based generator.
+__device__ __forceinline__ uint32_t mix32(uint32_t x) {
+  x ^= x >> 16; x *= 0x7feb352du;
+  x ^= x >> 15; x *= 0x846ca68bu;
+  x ^= x >> 16;
+  return x;
+}
+
+// Entry e of the Gaussian test matrix Omega of Algorithm 1 (Box-Muller on two
+// counter-derived uniforms); the same matrix for every user and every call.
+__device__ __forceinline__ float omega_entry(uint32_t e) {
+  const float u1 = ((float)(mix32(2u * e + 0x9e3779b9u) >> 8) + 0.5f) * (1.f / 16777216.f);
+  const float u2 = ((float)(mix32(2u * e + 0x85ebca6bu) >> 8) + 0.5f) * (1.f / 16777216.f);
+  return sqrtf(-2.f * __logf(u1)) * __cosf(6.2831853f * u2);
+}
+
+// 1/sqrt(x) in double from the fp32 approximation and two Newton steps.
+__device__ __forceinline__ double rsqrt_f64(double x) {
+  double y = (double)rsqrtf((float)x);
+  y = y * fma(-0.5 * x, y * y, 1.5);
+  y = y * fma(-0.5 * x, y * y, 1.5);
+  return y;
+}
+
+// ---- small dense products in shared memory -------------------------------------------
+
+// Out[D][p] = G Z.  G is [D][LD] (symmetric), Z and Out are [D][p], p even.
+// Each thread owns a 4 x 2 tile: four 16-byte reads of G rows and four 8-byte
+// reads of Z feed 32 FMAs, so the loop is not bound by shared-memory issue.
+template <int D, int LD>
+__device__ __forceinline__ void mul_G(const float* __restrict__ G, const float* __restrict__ Z,
+                                      float* __restrict__ Out, int p, int tid, int nt) {
+  const int cp = p >> 1;
+  const int ntiles = (D / 4) * cp;
+  for (int t = tid; t < ntiles; t += nt) {
+    const int j0 = (t % cp) * 2, i0 = (t / cp) * 4;
+    float acc[4][2];
+#pragma unroll
+    for (int m = 0; m < 4; ++m) { acc[m][0] = 0.f; acc[m][1] = 0.f; }
+#pragma unroll 2
+    for (int k = 0; k < D; k += 4) {
+      float4 g[4];
+#pragma unroll
+      for (int m = 0; m < 4; ++m) g[m] = *reinterpret_cast<const float4*>(G + (i0 + m) * LD + k);
+      const float2 z0 = *reinterpret_cast<const float2*>(Z + (k + 0) * p + j0);
+      const float2 z1 = *reinterpret_cast<const float2*>(Z + (k + 1) * p + j0);
+      const float2 z2 = *reinterpret_cast<const float2*>(Z + (k + 2) * p + j0);
+      const float2 z3 = *reinterpret_cast<const float2*>(Z + (k + 3) * p + j0);
+#pragma unroll
+      for (int m = 0; m < 4; ++m) {
+        acc[m][0] = fmaf(g[m].x, z0.x, acc[m][0]); acc[m][1] = fmaf(g[m].x, z0.y, acc[m][1]);
+        acc[m][0] = fmaf(g[m].y, z1.x, acc[m][0]); acc[m][1] = fmaf(g[m].y, z1.y, acc[m][1]);
+        acc[m][0] = fmaf(g[m].z, z2.x, acc[m][0]); acc[m][1] = fmaf(g[m].z, z2.y, acc[m][1]);
+        acc[m][0] = fmaf(g[m].w, z3.x, acc[m][0]); acc[m][1] = fmaf(g[m].w, z3.y, acc[m][1]);
+      }
+    }
+#pragma unroll
+    for (int m = 0; m < 4; ++m)
+      *reinterpret_cast<float2*>(Out + (i0 + m) * p + j0) = make_float2(acc[m][0], acc[m][1]);
+  }
+}
+
+// Out[a][c] = sum_k X[k][a] Y[k][c] over the D rows; X, Y are [D][p]; Out is [p][ldo].
+// 2 x 2 tile per thread, accumulation in Acc (double for the Cholesky-QR Gram matrix).
+template <int D, typename Acc, typename OutT>
+__device__ __forceinline__ void mul_XtY(const float* __restrict__ X, const float* __restrict__ Y,
+                                        OutT* __restrict__ Out, int p, int ldo, int tid, int nt) {
+  const int cp = p >> 1;
+  for (int t = tid; t < cp * cp; t += nt) {
+    const int c0 = (t % cp) * 2, a0 = (t / cp) * 2;
+    Acc s00 = 0, s01 = 0, s10 = 0, s11 = 0;
+#pragma unroll 4
+    for (int k = 0; k < D; ++k) {
+      const float2 x = *reinterpret_cast<const float2*>(X + k * p + a0);
+      const float2 y = *reinterpret_cast<const float2*>(Y + k * p + c0);
+      s00 += (Acc)x.x * (Acc)y.x; s01 += (Acc)x.x * (Acc)y.y;
+      s10 += (Acc)x.y * (Acc)y.x; s11 += (Acc)x.y * (Acc)y.y;
+    }
+    Out[a0 * ldo + c0] = (OutT)s00;       Out[a0 * ldo + c0 + 1] = (OutT)s01;
+    Out[(a0 + 1) * ldo + c0] = (OutT)s10; Out[(a0 + 1) * ldo + c0 + 1] = (OutT)s11;
+  }
+}
+
+// Cholesky A = L L^T of the p x p matrix A (double, [p][ld], ld even; the lower triangle
+// is overwritten by L) fused with the inverse Li = L^{-1} ([p][ld], upper part zero), by
+// ONE warp.  Lane j owns row j of L and column j of Li.  Step k computes column k of L
+// (a dot of row j with row k) and row k of Li (a dot of row k of L with column j of Li):
+// both use the same broadcast row of L, so the inverse rides in the latency shadow of the
+// factorisation.  A numerically dependent column (pivot below 1e-10 of its original diagonal
+// entry) is deflated: its column of L and row of Li are zero, so Q gets a zero column there.
+// Returns false (uniformly) only for a non-finite pivot.
+__device__ __forceinline__ bool cholesky_inverse_warp(double* __restrict__ A,
+                                                      double* __restrict__ Li,
+                                                      double* __restrict__ dref, int p, int ld,
+                                                      int lane) {
+  const int j = lane < p ? lane : 0;        // surplus lanes shadow lane 0 and store nothing
+  const bool mine = lane < p;
+  const double* row = A + j * ld;
+  if (mine) dref[j] = row[j];                // original diagonal: the yardstick of the pivots
+  __syncwarp();
+  for (int k = 0; k < p; ++k) {
+    const double* rk = A + k * ld;
+    double c0 = row[k], c1 = 0.0;
+    double e0 = (j == k) ? 1.0 : 0.0, e1 = 0.0;
+    int i = 0;
+#pragma unroll 2
+    for (; i + 1 < k; i += 2) {
+      const double2 lk = *reinterpret_cast<const double2*>(rk + i);
+      const double2 lj = *reinterpret_cast<const double2*>(row + i);
+      const double x0 = Li[i * ld + j], x1 = Li[(i + 1) * ld + j];
+      c0 = fma(-lj.x, lk.x, c0); c1 = fma(-lj.y, lk.y, c1);
+      e0 = fma(-lk.x, x0, e0);   e1 = fma(-lk.y, x1, e1);
+    }
+    if (i < k) {
+      const double lk = rk[i];
+      c0 = fma(-row[i], lk, c0);
+      e0 = fma(-lk, Li[i * ld + j], e0);
+    }
+    const double c = c0 + c1;
+    const double piv = __shfl_sync(0xffffffffu, c, k);
+    const double ref = dref[k];
+    if (!(piv < 1e300)) return false;                    // NaN or overflow
+    // A column whose part orthogonal to the earlier ones is below 1e-5 of its length is
+    // rounding residue of a rank-deficient block: it is dropped (zero column of Q).
+    const double inv = (piv > 1e-10 * ref) ? rsqrt_f64(piv) : 0.0;
+    if (mine && j >= k) A[j * ld + k] = c * inv;
+    if (mine) Li[k * ld + j] = (j <= k) ? (e0 + e1) * inv : 0.0;
+    __syncwarp();
+  }
+  return true;
+}
+
+// Z[i][j] = sum_{k<=j} Y[i][k] Li[j][k]  (Z = Y L^{-T}: the Q factor of the Cholesky-QR).
+// Two rows per thread share each 16-byte read of Li.
+template <int D>
+__device__ __forceinline__ void apply_Linv_t(const float* __restrict__ Y,
+                                             const double* __restrict__ Li, float* __restrict__ Z,
+                                             int p, int ld, int tid, int nt) {
+  for (int t = tid; t < (D / 2) * p; t += nt) {
+    const int j = t % p, i0 = (t / p) * 2;
+    double s0 = 0.0, s1 = 0.0, u0 = 0.0, u1 = 0.0;
+#pragma unroll 4
+    for (int k = 0; k < p; k += 2) {      // Li[j][k] = 0 for k > j
+      const double2 l = *reinterpret_cast<const double2*>(Li + j * ld + k);
+      const float2 ya = *reinterpret_cast<const float2*>(Y + i0 * p + k);
+      const float2 yb = *reinterpret_cast<const float2*>(Y + (i0 + 1) * p + k);
+      s0 = fma((double)ya.x, l.x, s0); s1 = fma((double)ya.y, l.y, s1);
+      u0 = fma((double)yb.x, l.x, u0); u1 = fma((double)yb.y, l.y, u1);
+    }
+    Z[i0 * p + j] = (float)(s0 + s1);
+    Z[(i0 + 1) * p + j] = (float)(u0 + u1);
+  }
+}
+
+// acc[m] = sum_k X[i0+m][k] M[k][col], m = 0..R-1: R rows of X ([.][p], 16-byte reads)
+// against one column of M ([p][ldm]).
+template <int R>
+__device__ __forceinline__ void rows_dot_col(const float* __restrict__ X, const float* __restrict__ M,
+                                             int p, int ldm, int i0, int col, float (&acc)[R]) {
+#pragma unroll
+  for (int m = 0; m < R; ++m) acc[m] = 0.f;
+#pragma unroll 2
+  for (int k = 0; k < p; k += 4) {
+    const float m0 = M[(k + 0) * ldm + col], m1 = M[(k + 1) * ldm + col];
+    const float m2 = M[(k + 2) * ldm + col], m3 = M[(k + 3) * ldm + col];
+#pragma unroll
+    for (int m = 0; m < R; ++m) {
+      const float4 x = *reinterpret_cast<const float4*>(X + (i0 + m) * p + k);
+      acc[m] = fmaf(x.x, m0, acc[m]); acc[m] = fmaf(x.y, m1, acc[m]);
+      acc[m] = fmaf(x.z, m2, acc[m]); acc[m] = fmaf(x.w, m3, acc[m]);
+    }
+  }
+}
+
+// ---- Jacobi on the p x p Rayleigh-Ritz matrix ------------------------------------------
+// Run by the first jt = roundup((p/2)^2, 32) threads of the CTA (barrier id 1); thread
+// (I, J) of the (p/2) x (p/2) grid owns one 2x2 block per round.  T is double-buffered
+// in Tc/Tn ([p][lp]); W ([p][lp]) accumulates the rotations and must hold the identity
+// on entry.  flags[0..2] are sweep flags (zero on entry).  Returns the buffer that holds
+// the final matrix; *sweeps_out = sweeps used, negative if the cap was reached.
+__device__ __forceinline__ float* ritz_jacobi(float* Tc, float* Tn, float* W, int p, int lp,
+                                              float thr_abs2, float sweep_stop2,
+                                              volatile int* flags, int tid, int jt,
+                                              int* sweeps_out) {
+  const int hp = p >> 1;
+  const bool active = tid < hp * hp;
+  const int I = active ? tid / hp : 0, J = active ? tid % hp : 0;
+  float* w0 = W + 2 * I * lp;
+  float* w1 = w0 + lp;
+  int sweeps = -kMaxSweeps;
+  int ar, cr, ac, cc;
+  pair_start(I, p, ar, cr);
+  pair_start(J, p, ac, cc);
+  for (int sweep = 0; sweep < kMaxSweeps; ++sweep) {
+    if (tid == 0) flags[(sweep + 1) % 3] = 0;
+    bool worst = false;
+    for (int k = 0; k < p - 1; ++k) {
+      if (active) {
+        const int pr = min(ar, cr), qr = max(ar, cr), pc = min(ac, cc), qc = max(ac, cc);
+        const float* tp = Tc + pr * lp;
+        const float* tq = Tc + qr * lp;
+        const float* up = Tc + pc * lp;
+        bool big_r, big_c;
+        const Rot rr = jacobi_rot(tp[pr], tq[qr], tp[qr], thr_abs2, sweep_stop2, big_r);
+        const Rot rc = jacobi_rot(up[pc], Tc[qc * lp + qc], up[qc], thr_abs2, sweep_stop2, big_c);
+        worst |= big_c;
+        float x00 = tp[pc], x01 = tp[qc], x10 = tq[pc], x11 = tq[qc];
+        float w00 = w0[pc], w01 = w0[qc], w10 = w1[pc], w11 = w1[qc];
+        if (I == J) {                      // the pair's own diagonal block
+          const float tg = rc.t * x01;
+          x00 -= tg; x11 += tg;
+          if (rc.s != 0.f) { x01 = 0.f; x10 = 0.f; }
+        } else {
+          rot_apply(rc, x00, x01); rot_apply(rc, x10, x11);   // columns
+          rot_apply(rr, x00, x10); rot_apply(rr, x01, x11);   // rows
+        }
+        rot_apply(rc, w00, w01); rot_apply(rc, w10, w11);
+        float* np_ = Tn + pr * lp;
+        float* nq_ = Tn + qr * lp;
+        np_[pc] = x00; np_[qc] = x01; nq_[pc] = x10; nq_[qc] = x11;
+        w0[pc] = w00; w0[qc] = w01; w1[pc] = w10; w1[qc] = w11;
+        pair_next(I, p, ar, cr);
+        pair_next(J, p, ac, cc);
+      }
+      if (k == p - 2 && worst) flags[sweep % 3] = 1;
+      bar_named(1, jt);
+      float* t = Tc; Tc = Tn; Tn = t;
+    }
+    if (flags[sweep % 3] == 0) { sweeps = sweep + 1; break; }
+  }
+  *sweeps_out = sweeps;
+  return Tc;
+}
+
+// Ranks of lam[0..n) in descending order (ties: lower index first): order[rank] = index.
+__device__ __forceinline__ void rank_descending(const float* lam, int* order, int n, int tid) {
+  if (tid < n) {
+    const float li = lam[tid];
+    int rank = 0;
+    for (int j = 0; j < n; ++j) {
+      const float lj = lam[j];
+      rank += (lj > li) || (lj == li && j < tid);
+    }
+    order[rank] = tid;
+  }
+}
+
+// route_taken[b] = route | power steps << 8 | Jacobi sweeps << 16
+constexpr int kRouteSubspace = 1, kRouteFull = 2;
+
+template <int D>
+__global__ void __launch_bounds__(EigCfg<D>::THREADS, 1)
+eig_kernel(const float* __restrict__ gpart, int splits, int r, int p, int route, EigTol tol,
+           float* __restrict__ S, float* __restrict__ V, int* __restrict__ info,
+           int* __restrict__ route_taken) {
+  using Cfg = EigCfg<D>;
+  constexpr int PT = Cfg::PT, SIDE = Cfg::SIDE, LD = Cfg::LD, NT = Cfg::THREADS;
+  extern __shared__ __align__(16) float smem[];
+  float* Gc = smem;                 // current matrix
+  float* Gn = smem + D * LD;        // next matrix
+  float* Vm = smem + 2 * D * LD;    // accumulated rotations (eigenvectors in columns)
+  float* lam = smem + 3 * D * LD;   // [D] eigenvalues
+  int* order = reinterpret_cast<int*>(lam + D);   // [D] column holding the k-th largest eigenvalue
+  __shared__ float s_gmax;
+  __shared__ double s_trace;
+  __shared__ int s_flags[4];
+  __shared__ int s_sweeps;
+
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
+
+  // ---- G = sum of the slices' partial Grams, in slice order -----------------
+  const float4* gp = reinterpret_cast<const float4*>(gpart + (size_t)b * splits * D * D);
+  int bad = 0;
+  for (int e = tid; e < D * D / 4; e += NT) {
+    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+    int s = 0;
+    for (; s + 8 <= splits; s += 8) {          // eight independent loads in flight
+      float4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = __ldg(gp + (size_t)(s + u) * (D * D / 4) + e);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        a0 += (double)v[u].x; a1 += (double)v[u].y; a2 += (double)v[u].z; a3 += (double)v[u].w;
+      }
+    }
+    if (s < splits) {                           // the remaining 1..7 slices, still loaded together
+      float4 v[7];
+#pragma unroll
+      for (int u = 0; u < 7; ++u)
+        v[u] = (s + u < splits) ? __ldg(gp + (size_t)(s + u) * (D * D / 4) + e)
+                                : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int u = 0; u < 7; ++u) {
+        a0 += (double)v[u].x; a1 += (double)v[u].y; a2 += (double)v[u].z; a3 += (double)v[u].w;
+      }
+    }
+    const float4 g = make_float4((float)a0, (float)a1, (float)a2, (float)a3);
+    bad |= !(isfinite(g.x) && isfinite(g.y) && isfinite(g.z) && isfinite(g.w));
+    *reinterpret_cast<float4*>(Gc + (e / (D / 4)) * LD + (e % (D / 4)) * 4) = g;
+  }
+  if (tid < 4) s_flags[tid] = 0;
+  bad = __syncthreads_or(bad);
+  if (bad) {
+    const float qnan = __int_as_float(0x7fc00000);
+    for (int e = tid; e < D * r; e += NT) V[(size_t)b * D * r + e] = qnan;
+    for (int e = tid; e < r; e += NT) S[(size_t)b * r + e] = qnan;
+    if (tid == 0 && info) info[b] = SOLAR_INFO_NONFINITE;
+    if (tid == 0 && route_taken) route_taken[b] = 0;
+    return;
+  }
+  if (tid < 32) {
+    float m = 0.f;
+    double tr = 0.0;
+    for (int i = tid; i < D; i += 32) {
+      const float g = Gc[i * LD + i];
+      m = fmaxf(m, fabsf(g));
+      tr += (double)g;
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) {
+      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      tr += __shfl_xor_sync(0xffffffffu, tr, o);
+    }
+    if (tid == 0) { s_gmax = m; s_trace = tr; }
+  }
+  __syncthreads();
+  const float gmax = s_gmax;
+  // Power-of-two scale that brings the largest diagonal entry into [1, 2): everything
+  // below works on sc * G (exact), and the eigenvalues are divided by sc at the end.
+  const float sc = gmax > 0.f ? exp2f(-(float)max(-100, min(100, ilogbf(gmax)))) : 1.f;
+  for (int e = tid; e < D * D; e += NT) Gc[(e / D) * LD + (e % D)] *= sc;
+  __syncthreads();
+  const float thr_abs2 = (kTolAbs * gmax * sc) * (kTolAbs * gmax * sc);
+  const float stop2 = tol.sweep_stop * tol.sweep_stop;
+
+  // ======================= route (1): certified subspace iteration =======================
+  if (p > 0 && route != kRouteFull && gmax > 0.f) {
+    constexpr int LP = Cfg::LP, PM = Cfg::PMAX;
+    float* sub = Cfg::ALIAS ? Gn : smem + Cfg::FULL_FLOATS;
+    constexpr int LPD = Cfg::LPD;
+    double* Ad = reinterpret_cast<double*>(sub);          // [PM][LPD] Y^T Y, then its Cholesky factor
+    double* Li = Ad + PM * LPD;                           // [PM][LPD] inverse of the factor
+    double* dref = Li + PM * LPD;                         // [PM]      diagonal of Y^T Y
+    float* Zb = reinterpret_cast<float*>(dref + PM);      // [D][p]    orthonormal basis
+    float* Yb = Zb + D * PM;                              // [D][p]    G Z
+    float* Xb = Yb + D * PM;                              // [D][p]    scratch / Ritz vectors
+    float* Tc = Xb + D * PM;                              // [p][LP]
+    float* Tn = Tc + PM * LP;
+    float* Wm = Tn + PM * LP;
+    float* theta = Wm + PM * LP;                          // [p]
+    float* res2 = theta + PM;                             // [p]
+    int* ordp = reinterpret_cast<int*>(res2 + PM);        // [p]
+
+    for (int e = tid; e < D * p; e += NT) Zb[e] = omega_entry((uint32_t)e);
+    __syncthreads();
+
+    int iters = 0;
+    bool ok = true, have_vectors = false;
+    mul_G<D, LD>(Gc, Zb, Yb, p, tid, NT);          // Y = G Omega
+    __syncthreads();
+    for (int it = 0; it < kMaxSubspaceIters && ok; ++it) {
+      // Cholesky-QR of the power step's Y = G Z:  A = Y^T Y = L L^T,  Z = Y L^-T
+      mul_XtY<D, double, double>(Yb, Yb, Ad, p, LPD, tid, NT);
+      __syncthreads();
+      if (tid < 32) {
+        const bool pd = cholesky_inverse_warp(Ad, Li, dref, p, LPD, lane);
+        if (tid == 0) s_flags[3] = pd ? 0 : 1;
+      }
+      __syncthreads();
+      if (s_flags[3]) { ok = false; break; }
+      apply_Linv_t<D>(Yb, Li, Zb, p, LPD, tid, NT);
+      __syncthreads();
+      // next power step (kept in Yb), Rayleigh-Ritz matrix T = Z^T (G Z), block residual G Z - Z T
+      mul_G<D, LD>(Gc, Zb, Yb, p, tid, NT);
+      __syncthreads();
+      mul_XtY<D, float, float>(Zb, Yb, Tc, p, LP, tid, NT);
+      __syncthreads();
+      iters = it + 1;
+      if (it + 1 == kMaxSubspaceIters) break;
+      // ||G Z - Z T||_F^2, accumulated per warp then by shared-memory atomics
+      if (tid == 0) res2[0] = 0.f;
+      __syncthreads();
+      float part = 0.f;
+      for (int t = tid; t < (D / 4) * p; t += NT) {
+        const int j = t % p, i0 = (t / p) * 4;
+        float zt[4];
+        rows_dot_col<4>(Zb, Tc, p, LP, i0, j, zt);
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+          const float d = Yb[(i0 + m) * p + j] - zt[m];
+          part = fmaf(d, d, part);
+        }
+      }
+#pragma unroll
+      for (int o = 16; o; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+      if (lane == 0) atomicAdd(&res2[0], part);
+      __syncthreads();
+      float tmax = 0.f;
+      for (int k = 0; k < p; ++k) tmax = fmaxf(tmax, fabsf(Tc[k * LP + k]));
+      const bool settled = sqrtf(res2[0]) <= tol.floor_rel * tmax;
+      __syncthreads();
+      // with oversampling (p > r) the extra directions never settle: two steps are the rule
+      if (settled || (p > r && it >= 1)) break;
+    }
+
+    if (ok) {
+      // symmetrise T, W = I
+      for (int e = tid; e < p * p; e += NT) {
+        const int a = e / p, c = e % p;
+        Wm[a * LP + c] = (a == c) ? 1.f : 0.f;
+        if (a < c) {
+          const float t = 0.5f * (Tc[a * LP + c] + Tc[c * LP + a]);
+          Tn[a * LP + c] = t; Tn[c * LP + a] = t;
+        } else if (a == c) {
+          Tn[a * LP + a] = Tc[a * LP + a];
+        }
+      }
+      __syncthreads();
+      float tmax = 0.f;
+      for (int k = 0; k < p; ++k) tmax = fmaxf(tmax, fabsf(Tn[k * LP + k]));
+      const int hp = p >> 1;
+      const int jt = min(NT, (hp * hp + 31) & ~31);
+      float* Tf = Tn;
+      if (tid < jt) {
+        int sw;
+        Tf = ritz_jacobi(Tn, Tc, Wm, p, LP, (kTolAbs * tmax) * (kTolAbs * tmax), stop2, s_flags, tid, jt, &sw);
+        if (tid == 0) s_sweeps = sw;
+      }
+      __syncthreads();
+      // every thread needs the final buffer: the sweep count's parity decides it
+      {
+        const int sw = s_sweeps;
+        const int rounds = (sw < 0 ? kMaxSweeps : sw) * (p - 1);
+        Tf = (rounds & 1) ? Tc : Tn;
+      }
+      if (tid < p) { theta[tid] = Tf[tid * LP + tid]; res2[tid] = 0.f; }
+      __syncthreads();
+      rank_descending(theta, ordp, p, tid);
+      __syncthreads();
+
+      // Ritz vectors v = Z w and residuals G v - theta v of the r kept pairs
+      for (int t = tid; t < (D / 2) * p; t += NT) {
+        const int jr = t % p, i0 = (t / p) * 2;
+        if (jr < r) {
+          const int col = ordp[jr];
+          float v[2], gv[2];
+          rows_dot_col<2>(Zb, Wm, p, LP, i0, col, v);
+          rows_dot_col<2>(Yb, Wm, p, LP, i0, col, gv);
+          Xb[i0 * p + jr] = v[0];
+          Xb[(i0 + 1) * p + jr] = v[1];
+          const float th = theta[col];
+          const float rho0 = gv[0] - th * v[0], rho1 = gv[1] - th * v[1];
+          atomicAdd(&res2[jr], fmaf(rho0, rho0, rho1 * rho1));
+        }
+      }
+      __syncthreads();
+
+      // certification (see the file header); all quantities are of sc * G
+      int good = 1;
+      if (tid < r) {
+        double kept = 0.0, rf2 = 0.0;
+        for (int k = 0; k < r; ++k) { kept += (double)theta[ordp[k]]; rf2 += (double)res2[k]; }
+        const float tail = (float)fmax((double)sc * s_trace - kept, 0.0);  // bounds every other eigenvalue
+        const float th1 = theta[ordp[0]];
+        const float thi = theta[ordp[tid]];
+        const float thr_ = theta[ordp[r - 1]];
+        const float cut = thr_ - tail - 2.f * sqrtf((float)rf2);
+        float gap = (tid == r - 1) ? cut : thi - theta[ordp[tid + 1]];
+        if (tid > 0) gap = fminf(gap, theta[ordp[tid - 1]] - thi);
+        const float resn = sqrtf(res2[tid]);
+        good = (cut > 0.f) && (thi > 0.f) &&
+               (resn <= fmaxf(tol.eps_vec * gap, tol.floor_rel * th1));
+        if (!(resn == resn)) good = 0;
+      }
+      if (s_sweeps < 0) good = 0;          // Jacobi sweep cap reached
+      ok = __syncthreads_and(good);
+      have_vectors = true;
+    }
+
+    if (ok || (route == kRouteSubspace && have_vectors)) {
+      // sign gauge and output
+      float* sgn = res2;
+      if (tid < r) {
+        float best = -1.f, lead = 1.f;
+        for (int j = 0; j < D; ++j) {
+          const float v = Xb[j * p + tid];
+          if (fabsf(v) > best) { best = fabsf(v); lead = v; }   // strict: lowest index wins a tie
+        }
+        S[(size_t)b * r + tid] = sqrtf(fmaxf(theta[ordp[tid]], 0.f) / sc);
+        sgn[tid] = lead < 0.f ? -1.f : 1.f;
+      }
+      __syncthreads();
+      for (int e = tid; e < D * r; e += NT) {
+        const int j = e / r, i = e % r;
+        V[(size_t)b * D * r + e] = Xb[j * p + i] * sgn[i];
+      }
+      if (tid == 0) {
+        if (info) info[b] = ok ? 0 : SOLAR_INFO_NOT_CERTIFIED;
+        if (route_taken) {
+          const int sw = s_sweeps;
+          route_taken[b] = kRouteSubspace | (iters << 8) | ((sw < 0 ? kMaxSweeps : sw) << 16);
+        }
+      }
+      return;
+    }
+    __syncthreads();
+  }
+
+  // ============================ route (2): full d x d Jacobi ============================
+  const int tI = tid / SIDE, tJ = tid % SIDE;
+  for (int e = tid; e < D * D; e += NT) {
+    const int i = e / D, j = e % D;
+    Vm[i * LD + j] = (i == j) ? 1.f : 0.f;
+  }
+  if (tid < 3) s_flags[tid] = 0;
+  __syncthreads();
+  int converged = 0, sweeps_done = kMaxSweeps;
+  int ar[PT], cr[PT], ac[PT], cc[PT];
+#pragma unroll
+  for (int a = 0; a < PT; ++a) {
+    pair_start(tI + a * SIDE, D, ar[a], cr[a]);
+    pair_start(tJ + a * SIDE, D, ac[a], cc[a]);
+  }
+  for (int sweep = 0; sweep < kMaxSweeps; ++sweep) {
+    if (tid == 0) s_flags[(sweep + 1) % 3] = 0;
+    bool worst = false;
+    for (int k = 0; k < D - 1; ++k) {
+      int pr[PT], qr[PT], pc[PT], qc[PT];
+      Rot rr[PT], rc[PT];
+#pragma unroll
+      for (int a = 0; a < PT; ++a) {
+        bool big_r, big_c;
+        pr[a] = min(ar[a], cr[a]); qr[a] = max(ar[a], cr[a]);
+        pc[a] = min(ac[a], cc[a]); qc[a] = max(ac[a], cc[a]);
+        rr[a] = jacobi_rot(Gc[pr[a] * LD + pr[a]], Gc[qr[a] * LD + qr[a]], Gc[pr[a] * LD + qr[a]],
+                           thr_abs2, stop2, big_r);
+        rc[a] = jacobi_rot(Gc[pc[a] * LD + pc[a]], Gc[qc[a] * LD + qc[a]], Gc[pc[a] * LD + qc[a]],
+                           thr_abs2, stop2, big_c);
+        worst |= big_c;
+      }
+#pragma unroll
+      for (int a = 0; a < PT; ++a) {
+        const float* gp_ = Gc + pr[a] * LD;
+        const float* gq_ = Gc + qr[a] * LD;
+        float* np_ = Gn + pr[a] * LD;
+        float* nq_ = Gn + qr[a] * LD;
+        float* v0 = Vm + 2 * (tI + a * SIDE) * LD;    // V' = V J_col on fixed rows (2I, 2I+1)
+        float* v1 = v0 + LD;
+#pragma unroll
+        for (int c = 0; c < PT; ++c) {
+          // G' = J_row^T G J_col on the block rows (p,q) x columns (p',q')
+          float x00 = gp_[pc[c]], x01 = gp_[qc[c]], x10 = gq_[pc[c]], x11 = gq_[qc[c]];
+          float v00 = v0[pc[c]], v01 = v0[qc[c]], v10 = v1[pc[c]], v11 = v1[qc[c]];
+          if (pr[a] == pc[c]) {            // the pair's own diagonal block
+            const float tg = rc[c].t * x01;
+            x00 -= tg; x11 += tg;
+            if (rc[c].s != 0.f) { x01 = 0.f; x10 = 0.f; }
+          } else {
+            rot_apply(rc[c], x00, x01); rot_apply(rc[c], x10, x11);   // columns
+            rot_apply(rr[a], x00, x10); rot_apply(rr[a], x01, x11);   // rows
+          }
+          rot_apply(rc[c], v00, v01); rot_apply(rc[c], v10, v11);
+          np_[pc[c]] = x00; np_[qc[c]] = x01; nq_[pc[c]] = x10; nq_[qc[c]] = x11;
+          v0[pc[c]] = v00; v0[qc[c]] = v01; v1[pc[c]] = v10; v1[qc[c]] = v11;
+        }
+      }
+#pragma unroll
+      for (int a = 0; a < PT; ++a) {
+        pair_next(tI + a * SIDE, D, ar[a], cr[a]);
+        pair_next(tJ + a * SIDE, D, ac[a], cc[a]);
+      }
+      if (k == D - 2 && worst) s_flags[sweep % 3] = 1;
+      __syncthreads();
+      float* t = Gc; Gc = Gn; Gn = t;
+    }
+    if (s_flags[sweep % 3] == 0) { converged = 1; sweeps_done = sweep + 1; break; }
+  }
+
+  // ---- order the eigenvalues, keep r, fix the sign of each vector ----------------
+  if (tid < D) lam[tid] = Gc[tid * LD + tid];
+  __syncthreads();
+  rank_descending(lam, order, D, tid);
+  __syncthreads();
+  float* sgn = Gn;   // reuse: [r] signs
+  if (tid < r) {
+    const int col = order[tid];
+    float best = -1.f, lead = 1.f;
+    for (int j = 0; j < D; ++j) {
+      const float v = Vm[j * LD + col];
+      if (fabsf(v) > best) { best = fabsf(v); lead = v; }   // strict: lowest index wins a tie
+    }
+    sgn[tid] = lead < 0.f ? -1.f : 1.f;
+    S[(size_t)b * r + tid] = sqrtf(fmaxf(lam[col], 0.f) / sc);
+  }
+  __syncthreads();
+  for (int e = tid; e < D * r; e += NT) {
+    const int j = e / r, i = e % r;
+    V[(size_t)b * D * r + e] = Vm[j * LD + order[i]] * sgn[i];
+  }
+  if (tid == 0) {
+    if (info) info[b] = converged ? 0 : SOLAR_INFO_NOT_CONVERGED;
+    if (route_taken) route_taken[b] = kRouteFull | (sweeps_done << 16);
+  }
+}
+
+template <int D>
+cudaError_t launch_d(int B, int r, int p, int route, EigTol tol, const float* gpart, int splits,
+                     float* S, float* V, int* info, int* route_taken, cudaStream_t st) {
+  using Cfg = EigCfg<D>;
+  if (p > Cfg::PMAX) p = 0;
+  cudaError_t e = cudaFuncSetAttribute(eig_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)Cfg::SMEM);
+  if (e != cudaSuccess) return e;
+  eig_kernel<D><<<B, Cfg::THREADS, Cfg::SMEM, st>>>(gpart, splits, r, p, route, tol, S, V, info,
+                                                    route_taken);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+// Subspace dimension for rank r in width d: r rounded up to a multiple of 8 (a little
+// oversampling; surplus directions of an exactly rank-r input deflate), if that is at most
+// min(32, d/2); otherwise 0: the subspace route brings nothing.
+int eig_subspace_dim(int d, int r) {
+  const int p = (r + 7) / 8 * 8;
+  return (p <= 32 && 2 * p <= d) ? p : 0;
+}
+
+cudaError_t launch_eig(int B, int d, int r, solar_dtype_t dt, int route, const float* gpart,
+                       int splits, float* S, float* V, int* info, int* route_taken,
+                       cudaStream_t st) {
+  EigTol tol;
+  if (dt == SOLAR_BF16) {
+    tol.eps_vec = 1e-3f; tol.floor_rel = 256.f * kUnit; tol.sweep_stop = 1e-4f;
+  } else {
+    tol.eps_vec = 1e-5f; tol.floor_rel = 32.f * kUnit; tol.sweep_stop = 1e-5f;
+  }
+  const int p = eig_subspace_dim(d, r);
+  switch (d) {
+    case 32: return launch_d<32>(B, r, p, route, tol, gpart, splits, S, V, info, route_taken, st);
+    case 64: return launch_d<64>(B, r, p, route, tol, gpart, splits, S, V, info, route_taken, st);
+    case 128: return launch_d<128>(B, r, p, route, tol, gpart, splits, S, V, info, route_taken, st);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+}  // namespace solar

@@ -72,18 +72,29 @@ solar_status_t solar_gram_partials(int B, int N, int d, solar_dtype_t dt, const 
                                     static_cast<cudaStream_t>(stream)));
 }
 
-solar_status_t solar_eig_from_partials(int B, int N, int d, int r, solar_dtype_t dt, float* S,
-                                       float* V, int* info, void* workspace,
-                                       size_t workspace_bytes, void* stream) {
+solar_status_t solar_eig_from_partials_ex(int B, int N, int d, int r, solar_dtype_t dt, int route,
+                                          float* S, float* V, int* info, int* route_taken,
+                                          void* workspace, size_t workspace_bytes, void* stream) {
   SOLAR_TRY(check_dims(B, 0, N, d, r, dt));
+  if (route != SOLAR_ROUTE_AUTO && route != SOLAR_ROUTE_SUBSPACE && route != SOLAR_ROUTE_FULL)
+    return SOLAR_ERR_INVALID_ARG;
   if (B == 0) return SOLAR_OK;
   SOLAR_TRY(check_ptr(S));
   SOLAR_TRY(check_ptr(V));
   if (info != nullptr && (reinterpret_cast<uintptr_t>(info) & 3u)) return SOLAR_ERR_INVALID_ARG;
+  if (route_taken != nullptr && (reinterpret_cast<uintptr_t>(route_taken) & 3u))
+    return SOLAR_ERR_INVALID_ARG;
   SOLAR_TRY(check_ws(workspace, workspace_bytes, factor_ws_bytes(B, N, d)));
   const GramPlan plan = gram_plan(B, N);
-  return from_cuda(launch_eig_jacobi(B, d, r, static_cast<const float*>(workspace), plan.splits, S,
-                                     V, info, static_cast<cudaStream_t>(stream)));
+  return from_cuda(launch_eig(B, d, r, dt, route, static_cast<const float*>(workspace), plan.splits,
+                              S, V, info, route_taken, static_cast<cudaStream_t>(stream)));
+}
+
+solar_status_t solar_eig_from_partials(int B, int N, int d, int r, solar_dtype_t dt, float* S,
+                                       float* V, int* info, void* workspace,
+                                       size_t workspace_bytes, void* stream) {
+  return solar_eig_from_partials_ex(B, N, d, r, dt, SOLAR_ROUTE_AUTO, S, V, info, nullptr,
+                                    workspace, workspace_bytes, stream);
 }
 
 solar_status_t solar_project_us(int B, int N, int d, int r, solar_dtype_t dt, const void* H,

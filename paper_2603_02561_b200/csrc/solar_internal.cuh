@@ -79,8 +79,10 @@ inline size_t attn_ws_bytes(int B, int d, int r) {
 // ---- launchers (one per kernel file) --------------------------------------
 cudaError_t launch_gram_simt(int B, int N, int d, solar_dtype_t dt, const void* H, float* gpart,
                              const GramPlan& plan, cudaStream_t st);
-cudaError_t launch_eig_jacobi(int B, int d, int r, const float* gpart, int splits, float* S,
-                              float* V, int* info, cudaStream_t st);
+cudaError_t launch_eig(int B, int d, int r, solar_dtype_t dt, int route, const float* gpart,
+                       int splits, float* S, float* V, int* info, int* route_taken,
+                       cudaStream_t st);
+int eig_subspace_dim(int d, int r);
 cudaError_t launch_project_us(int B, int N, int d, int r, solar_dtype_t dt, const void* H,
                               const float* V, void* US, cudaStream_t st);
 cudaError_t launch_attn_prepare(int B, int d, int r, solar_dtype_t dt, const float* S,

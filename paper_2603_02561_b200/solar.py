@@ -17,7 +17,8 @@ LIB_PATH = os.path.join(_HERE, "libsolar_b200.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA = range(5)
 F32, BF16 = 0, 1
 FLAG_NO_SOFTMAX = 1
-INFO_NOT_CONVERGED, INFO_NONFINITE = 1, 2
+INFO_NOT_CONVERGED, INFO_NONFINITE, INFO_NOT_CERTIFIED = 1, 2, 4
+ROUTE_AUTO, ROUTE_SUBSPACE, ROUTE_FULL = 0, 1, 2
 
 _c_int, _c_size, _c_vp, _c_float, _c_uint = (ctypes.c_int, ctypes.c_size_t, ctypes.c_void_p,
                                               ctypes.c_float, ctypes.c_uint)
@@ -32,6 +33,8 @@ SIGNATURES = {
     "solar_gram_splits": (_c_int, [_c_int] * 3 + [_c_int]),
     "solar_gram_partials": (_c_int, [_c_int] * 3 + [_c_int, _c_vp, _c_vp, _c_size, _c_vp]),
     "solar_eig_from_partials": (_c_int, [_c_int] * 4 + [_c_int] + [_c_vp] * 3 + [_c_vp, _c_size, _c_vp]),
+    "solar_eig_from_partials_ex": (_c_int, [_c_int] * 4 + [_c_int, _c_int] + [_c_vp] * 4 +
+                                   [_c_vp, _c_size, _c_vp]),
     "solar_project_us": (_c_int, [_c_int] * 4 + [_c_int] + [_c_vp] * 3 + [_c_vp]),
     "solar_attn_prepare": (_c_int, [_c_int] * 3 + [_c_int] + [_c_vp] * 5 + [_c_float, _c_vp, _c_size, _c_vp]),
     "solar_static_scratch_bytes": (_c_size, []),
@@ -179,6 +182,13 @@ def eig_from_partials(B, N, d, r, dtype, S, V, info, workspace, stream=None):
     _check(lib().solar_eig_from_partials(B, N, d, r, dtype_code(dtype), _ptr(S), _ptr(V), _ptr(info),
                                          _ptr(workspace), workspace.numel(), _stream(stream)),
            "solar_eig_from_partials")
+
+
+def eig_from_partials_ex(B, N, d, r, dtype, route, S, V, info, route_taken, workspace, stream=None):
+    _check(lib().solar_eig_from_partials_ex(B, N, d, r, dtype_code(dtype), int(route), _ptr(S), _ptr(V),
+                                            _ptr(info), _ptr(route_taken), _ptr(workspace),
+                                            workspace.numel(), _stream(stream)),
+           "solar_eig_from_partials_ex")
 
 
 def project_us(H, V, US, stream=None):
