@@ -55,8 +55,10 @@ enum {
 enum {
   SOLAR_INFO_NOT_CONVERGED = 1, /* sweep cap reached before every rotation became negligible */
   SOLAR_INFO_NONFINITE = 2,     /* H_b^T H_b contains NaN or Inf; s, V of this user are NaN  */
-  SOLAR_INFO_NOT_CERTIFIED = 4  /* only with SOLAR_ROUTE_SUBSPACE: the range-finder result was
+  SOLAR_INFO_NOT_CERTIFIED = 4, /* only with SOLAR_ROUTE_SUBSPACE: the range-finder result was
                                    written although its error bounds did not hold              */
+  SOLAR_INFO_DEVICE_WAIT = 8    /* a bounded wait inside the Gram kernel (on a TMA copy or on the
+                                   tensor cores) ran out; s, V of this user are NaN             */
 };
 
 /* How solar_eig_from_partials_ex reaches the top-r eigenpairs of H_b^T H_b.
@@ -133,8 +135,11 @@ int solar_gram_splits(int B, int N, int d, solar_dtype_t dt);
 
 /* Streaming pass over H: slice s of user b contributes the d x d partial Gram
  *   P[b,s] = sum over the rows n of slice s of h_n h_n^T        (fp32)
- * stored at ((float*)workspace)[(b*splits + s)*d*d ...], row-major.
- * H_b^T H_b (the matrix whose eigenvectors are V of Eq. 9) is the sum over s. */
+ * stored at ((float*)workspace)[(b*splits + s)*d*d ...], row-major; the kernel's
+ * per-slice status words follow the partials (read by solar_eig_from_partials).
+ * H_b^T H_b (the matrix whose eigenvectors are V of Eq. 9) is the sum over s.
+ * bf16 storage with d = 64 or 128 and N >= 128 runs on the tensor cores (TMA tiles,
+ * tcgen05.mma, fp32 accumulation in tensor memory); other shapes use FFMA. */
 solar_status_t solar_gram_partials(int B, int N, int d, solar_dtype_t dt, const void* H,
                                    void* workspace, size_t workspace_bytes, void* stream);
 

@@ -3,9 +3,14 @@
 //   Value_r = (V Sigma)^T W_V   [r,d]
 // and the folded score operand T_b = scale * W_Q Key_r^T [d,r], so that the
 // scores of Eq. 12 are  scale * (C W_Q) Key_r^T = C T_b.
-// Written to the workspace in fp32 and as bf16 operand images for the
-// tensor-core attention kernel (T^T split into a high and a low bf16 half so
-// that the score GEMM keeps ~16 mantissa bits; Value_r^T).
+// Written to the workspace in fp32 (for the FFMA attention kernel) and as packed bf16
+// operand images for the tensor-core attention kernel: T^T and Value_r^T, each split
+// into a high and a low bf16 half so that both GEMMs keep ~16 mantissa bits, zero padded
+// to 64 token slots.
+//
+// One CTA per user.  Each weight matrix is staged once in shared memory with coalesced
+// 16-byte loads; the three small products then run out of shared memory with 4 outputs
+// per thread.
 #include "solar_internal.cuh"
 
 namespace solar {
@@ -14,53 +19,116 @@ namespace {
 
 constexpr int kPrepThreads = 512;
 
+// Stages W[D][D] (storage type T) as fp32 in shared memory.
+template <typename T, int D>
+__device__ __forceinline__ void stage_weight(const T* __restrict__ W, float* __restrict__ Ws, int tid) {
+  constexpr int VE = Vec16<T>::kElems;
+  for (int v = tid; v < D * D / VE; v += kPrepThreads) {
+    float tmp[VE];
+    Vec16<T>::load(W + (size_t)v * VE, tmp);
+#pragma unroll
+    for (int e = 0; e < VE; ++e) Ws[v * VE + e] = tmp[e];
+  }
+}
+
 template <typename T, int D>
 __global__ void __launch_bounds__(kPrepThreads)
 attn_prepare_kernel(const float* __restrict__ S, const float* __restrict__ V,
                     const T* __restrict__ Wq, const T* __restrict__ Wk, const T* __restrict__ Wv,
                     float scale, int r, char* __restrict__ ws, AttnWs lay) {
-  extern __shared__ float sm[];
-  float* VS = sm;            // [D][r]   V Sigma
-  float* KrT = sm + D * r;   // [D][r]   Key_r^T
+  extern __shared__ __align__(16) float sm[];
+  const int rp = (r + 3) & ~3;          // token pitch: rows of VS / KrT are read 4 at a time
+  float* Ws = sm;                       // [D][D]   the weight matrix in use
+  float* VS = Ws + D * D;               // [D][rp]  V Sigma (zero in the padding)
+  float* KrT = VS + D * rp;             // [D][rp]  Key_r^T
   const int b = blockIdx.x, tid = threadIdx.x;
   char* wsb = ws + (size_t)b * lay.per_user;
   float* Tf = reinterpret_cast<float*>(wsb + lay.tf_off);
   float* Vr = reinterpret_cast<float*>(wsb + lay.vr_off);
-  __nv_bfloat16* Thi = reinterpret_cast<__nv_bfloat16*>(wsb + lay.thi_off);
-  __nv_bfloat16* Tlo = reinterpret_cast<__nv_bfloat16*>(wsb + lay.tlo_off);
-  __nv_bfloat16* VrT = reinterpret_cast<__nv_bfloat16*>(wsb + lay.vrt_off);
+  __nv_bfloat16* Tpk = reinterpret_cast<__nv_bfloat16*>(wsb + lay.tpk_off);
+  __nv_bfloat16* Vpk = reinterpret_cast<__nv_bfloat16*>(wsb + lay.vpk_off);
+  const __nv_bfloat16 zero = __float2bfloat16_rn(0.f);
 
-  for (int e = tid; e < D * r; e += kPrepThreads)
-    VS[e] = V[(size_t)b * D * r + e] * S[(size_t)b * r + (e % r)];
-  __syncthreads();
-
-  // Key_r[i][j] = sum_k VS[k][i] Wk[k][j];  Value_r likewise with Wv.
-  for (int e = tid; e < D * r; e += kPrepThreads) {
-    const int i = e / D, j = e % D;          // j fastest: coalesced weight reads
-    float ak = 0.f, av = 0.f;
-#pragma unroll 8
-    for (int k = 0; k < D; ++k) {
-      const float vs = VS[k * r + i];
-      ak = fmaf(vs, to_f32<T>(Wk[k * D + j]), ak);
-      av = fmaf(vs, to_f32<T>(Wv[k * D + j]), av);
-    }
-    KrT[j * r + i] = ak;
-    Vr[i * D + j] = av;
-    VrT[j * r + i] = __float2bfloat16_rn(av);
+  stage_weight<T, D>(Wk, Ws, tid);
+  for (int e = tid; e < D * rp; e += kPrepThreads) {
+    const int k = e / rp, i = e % rp;
+    VS[e] = i < r ? V[((size_t)b * D + k) * r + i] * S[(size_t)b * r + i] : 0.f;
+  }
+  // zero padding of the packed operands: token slots r .. 63
+  for (int e = tid; e < 2 * (kTokenSlots - r) * D; e += kPrepThreads) {
+    const int h = e / ((kTokenSlots - r) * D), rem = e % ((kTokenSlots - r) * D);
+    Tpk[((size_t)h * kTokenSlots + r) * D + rem] = zero;
+  }
+  for (int e = tid; e < 2 * D * (kTokenSlots - r); e += kPrepThreads) {
+    const int row = e / (kTokenSlots - r), i = r + e % (kTokenSlots - r);
+    Vpk[(size_t)row * kTokenSlots + i] = zero;      // row runs over [2][D]
   }
   __syncthreads();
 
-  // T[k][i] = scale * sum_j Wq[k][j] Key_r[i][j]
-  for (int e = tid; e < D * r; e += kPrepThreads) {
-    const int k = e / r, i = e % r;          // i fastest: conflict-free KrT reads
-    float acc = 0.f;
+  // X[i][j] = sum_k VS[k][i] W[k][j] for four tokens i per thread; j runs along the lanes.
+  auto project = [&](float (&acc)[4], int i0, int j) {
+#pragma unroll
+    for (int m = 0; m < 4; ++m) acc[m] = 0.f;
 #pragma unroll 8
-    for (int j = 0; j < D; ++j) acc = fmaf(to_f32<T>(Wq[k * D + j]), KrT[j * r + i], acc);
-    acc *= scale;
-    Tf[k * r + i] = acc;
-    const __nv_bfloat16 hi = __float2bfloat16_rn(acc);
-    Thi[i * D + k] = hi;
-    Tlo[i * D + k] = __float2bfloat16_rn(acc - __bfloat162float(hi));
+    for (int k = 0; k < D; ++k) {
+      const float w = Ws[k * D + j];
+      const float4 vs = *reinterpret_cast<const float4*>(VS + k * rp + i0);
+      acc[0] = fmaf(vs.x, w, acc[0]); acc[1] = fmaf(vs.y, w, acc[1]);
+      acc[2] = fmaf(vs.z, w, acc[2]); acc[3] = fmaf(vs.w, w, acc[3]);
+    }
+  };
+
+  // Key_r^T
+  for (int t = tid; t < (rp / 4) * D; t += kPrepThreads) {
+    const int j = t % D, i0 = (t / D) * 4;
+    float acc[4];
+    project(acc, i0, j);
+    *reinterpret_cast<float4*>(KrT + j * rp + i0) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+  }
+  __syncthreads();
+  stage_weight<T, D>(Wv, Ws, tid);
+  __syncthreads();
+  // Value_r (fp32) and Value_r^T (packed bf16 halves)
+  for (int t = tid; t < (rp / 4) * D; t += kPrepThreads) {
+    const int j = t % D, i0 = (t / D) * 4;
+    float acc[4];
+    project(acc, i0, j);
+#pragma unroll
+    for (int m = 0; m < 4; ++m) {
+      const int i = i0 + m;
+      if (i < r) {
+        Vr[i * D + j] = acc[m];
+        const __nv_bfloat16 hi = __float2bfloat16_rn(acc[m]);
+        Vpk[(size_t)j * kTokenSlots + i] = hi;
+        Vpk[(size_t)(D + j) * kTokenSlots + i] = __float2bfloat16_rn(acc[m] - __bfloat162float(hi));
+      }
+    }
+  }
+  __syncthreads();
+  stage_weight<T, D>(Wq, Ws, tid);
+  __syncthreads();
+  // T[k][i] = scale * sum_j Wq[k][j] Key_r[i][j], four tokens i per thread
+  for (int t = tid; t < (rp / 4) * D; t += kPrepThreads) {
+    const int i0 = (t % (rp / 4)) * 4, k = t / (rp / 4);
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 8
+    for (int j = 0; j < D; ++j) {
+      const float w = Ws[k * D + j];
+      const float4 kr = *reinterpret_cast<const float4*>(KrT + j * rp + i0);
+      acc[0] = fmaf(w, kr.x, acc[0]); acc[1] = fmaf(w, kr.y, acc[1]);
+      acc[2] = fmaf(w, kr.z, acc[2]); acc[3] = fmaf(w, kr.w, acc[3]);
+    }
+#pragma unroll
+    for (int m = 0; m < 4; ++m) {
+      const int i = i0 + m;
+      if (i < r) {
+        const float v = acc[m] * scale;
+        Tf[k * r + i] = v;
+        const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+        Tpk[(size_t)i * D + k] = hi;
+        Tpk[((size_t)kTokenSlots + i) * D + k] = __float2bfloat16_rn(v - __bfloat162float(hi));
+      }
+    }
   }
 }
 
@@ -68,7 +136,8 @@ template <typename T>
 cudaError_t launch_t(int B, int d, int r, const float* S, const float* V, const void* Wq,
                      const void* Wk, const void* Wv, float scale, char* ws, const AttnWs& lay,
                      cudaStream_t st) {
-  const size_t smem = (size_t)2 * d * r * sizeof(float);
+  const int rp = (r + 3) & ~3;
+  const size_t smem = (size_t)(d * d + 2 * d * rp) * sizeof(float);
   const T* q = static_cast<const T*>(Wq);
   const T* k = static_cast<const T*>(Wk);
   const T* v = static_cast<const T*>(Wv);

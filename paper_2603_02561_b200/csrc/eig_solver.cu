@@ -382,9 +382,9 @@ constexpr int kRouteSubspace = 1, kRouteFull = 2;
 
 template <int D>
 __global__ void __launch_bounds__(EigCfg<D>::THREADS, 1)
-eig_kernel(const float* __restrict__ gpart, int splits, int r, int p, int route, EigTol tol,
-           float* __restrict__ S, float* __restrict__ V, int* __restrict__ info,
-           int* __restrict__ route_taken) {
+eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status, int splits, int r,
+           int p, int route, EigTol tol, float* __restrict__ S, float* __restrict__ V,
+           int* __restrict__ info, int* __restrict__ route_taken) {
   using Cfg = EigCfg<D>;
   constexpr int PT = Cfg::PT, SIDE = Cfg::SIDE, LD = Cfg::LD, NT = Cfg::THREADS;
   extern __shared__ __align__(16) float smem[];
@@ -431,12 +431,16 @@ eig_kernel(const float* __restrict__ gpart, int splits, int r, int p, int route,
     *reinterpret_cast<float4*>(Gc + (e / (D / 4)) * LD + (e % (D / 4)) * 4) = g;
   }
   if (tid < 4) s_flags[tid] = 0;
+  // a Gram CTA whose bounded wait ran out leaves a code other than kGramStatusOk
+  int lost = 0;
+  for (int s = tid; s < splits; s += NT) lost |= (gram_status[b * splits + s] != kGramStatusOk);
+  lost = __syncthreads_or(lost);
   bad = __syncthreads_or(bad);
-  if (bad) {
+  if (bad || lost) {
     const float qnan = __int_as_float(0x7fc00000);
     for (int e = tid; e < D * r; e += NT) V[(size_t)b * D * r + e] = qnan;
     for (int e = tid; e < r; e += NT) S[(size_t)b * r + e] = qnan;
-    if (tid == 0 && info) info[b] = SOLAR_INFO_NONFINITE;
+    if (tid == 0 && info) info[b] = lost ? SOLAR_INFO_DEVICE_WAIT : SOLAR_INFO_NONFINITE;
     if (tid == 0 && route_taken) route_taken[b] = 0;
     return;
   }
@@ -736,15 +740,16 @@ eig_kernel(const float* __restrict__ gpart, int splits, int r, int p, int route,
 }
 
 template <int D>
-cudaError_t launch_d(int B, int r, int p, int route, EigTol tol, const float* gpart, int splits,
-                     float* S, float* V, int* info, int* route_taken, cudaStream_t st) {
+cudaError_t launch_d(int B, int r, int p, int route, EigTol tol, const float* gpart,
+                     const int* gram_status, int splits, float* S, float* V, int* info,
+                     int* route_taken, cudaStream_t st) {
   using Cfg = EigCfg<D>;
   if (p > Cfg::PMAX) p = 0;
   cudaError_t e = cudaFuncSetAttribute(eig_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)Cfg::SMEM);
   if (e != cudaSuccess) return e;
-  eig_kernel<D><<<B, Cfg::THREADS, Cfg::SMEM, st>>>(gpart, splits, r, p, route, tol, S, V, info,
-                                                    route_taken);
+  eig_kernel<D><<<B, Cfg::THREADS, Cfg::SMEM, st>>>(gpart, gram_status, splits, r, p, route, tol, S,
+                                                    V, info, route_taken);
   return cudaGetLastError();
 }
 
@@ -759,8 +764,8 @@ int eig_subspace_dim(int d, int r) {
 }
 
 cudaError_t launch_eig(int B, int d, int r, solar_dtype_t dt, int route, const float* gpart,
-                       int splits, float* S, float* V, int* info, int* route_taken,
-                       cudaStream_t st) {
+                       const int* gram_status, int splits, float* S, float* V, int* info,
+                       int* route_taken, cudaStream_t st) {
   EigTol tol;
   if (dt == SOLAR_BF16) {
     tol.eps_vec = 1e-3f; tol.floor_rel = 256.f * kUnit; tol.sweep_stop = 1e-4f;
@@ -769,9 +774,9 @@ cudaError_t launch_eig(int B, int d, int r, solar_dtype_t dt, int route, const f
   }
   const int p = eig_subspace_dim(d, r);
   switch (d) {
-    case 32: return launch_d<32>(B, r, p, route, tol, gpart, splits, S, V, info, route_taken, st);
-    case 64: return launch_d<64>(B, r, p, route, tol, gpart, splits, S, V, info, route_taken, st);
-    case 128: return launch_d<128>(B, r, p, route, tol, gpart, splits, S, V, info, route_taken, st);
+    case 32: return launch_d<32>(B, r, p, route, tol, gpart, gram_status, splits, S, V, info, route_taken, st);
+    case 64: return launch_d<64>(B, r, p, route, tol, gpart, gram_status, splits, S, V, info, route_taken, st);
+    case 128: return launch_d<128>(B, r, p, route, tol, gpart, gram_status, splits, S, V, info, route_taken, st);
     default: return cudaErrorInvalidValue;
   }
 }

@@ -1,14 +1,15 @@
 // Streaming Gram pass, FFMA version: P[b,s] = sum_{n in slice s} h_n h_n^T.
-// Used for fp32 storage and for d = 32 (shapes the tensor-core kernel does not
-// take); G_b = H_b^T H_b is the matrix whose eigenvectors are V of Eq. 9.
+// Used for fp32 storage (bf16 products would break the 1e-4 tolerance of that mode),
+// for d = 32 and for N < 128 (shapes the tensor-core kernel does not take);
+// G_b = H_b^T H_b is the matrix whose eigenvectors are V of Eq. 9.
 #include "solar_internal.cuh"
 
 namespace solar {
 
 template <typename T, int D>
 __global__ void __launch_bounds__(256)
-gram_simt_kernel(const T* __restrict__ H, float* __restrict__ gpart, int N, int chunk_rows,
-                 int splits) {
+gram_simt_kernel(const T* __restrict__ H, float* __restrict__ gpart, int* __restrict__ status,
+                 int N, int chunk_rows, int splits) {
   constexpr int TR = 32;      // rows staged per step
   constexpr int R = D / 16;   // each thread owns an R x R register tile of G
   __shared__ float tile[TR][D];
@@ -61,27 +62,28 @@ gram_simt_kernel(const T* __restrict__ H, float* __restrict__ gpart, int N, int 
   for (int i = 0; i < R; ++i)
 #pragma unroll
     for (int j = 0; j < R; ++j) out[(ty + 16 * i) * D + tx + 16 * j] = acc[i][j];
+  if (threadIdx.x == 0) status[b * splits + s] = kGramStatusOk;   // this kernel has no waits to lose
 }
 
 template <typename T>
-static cudaError_t launch_t(int B, int N, int d, const void* H, float* gpart, const GramPlan& plan,
-                            cudaStream_t st) {
+static cudaError_t launch_t(int B, int N, int d, const void* H, float* gpart, int* status,
+                            const GramPlan& plan, cudaStream_t st) {
   const dim3 grid(plan.splits, B), block(256);
   const int chunk_rows = plan.chunk_tiles * kGramTileRows;
   const T* h = static_cast<const T*>(H);
   switch (d) {
-    case 32: gram_simt_kernel<T, 32><<<grid, block, 0, st>>>(h, gpart, N, chunk_rows, plan.splits); break;
-    case 64: gram_simt_kernel<T, 64><<<grid, block, 0, st>>>(h, gpart, N, chunk_rows, plan.splits); break;
-    case 128: gram_simt_kernel<T, 128><<<grid, block, 0, st>>>(h, gpart, N, chunk_rows, plan.splits); break;
+    case 32: gram_simt_kernel<T, 32><<<grid, block, 0, st>>>(h, gpart, status, N, chunk_rows, plan.splits); break;
+    case 64: gram_simt_kernel<T, 64><<<grid, block, 0, st>>>(h, gpart, status, N, chunk_rows, plan.splits); break;
+    case 128: gram_simt_kernel<T, 128><<<grid, block, 0, st>>>(h, gpart, status, N, chunk_rows, plan.splits); break;
     default: return cudaErrorInvalidValue;
   }
   return cudaGetLastError();
 }
 
 cudaError_t launch_gram_simt(int B, int N, int d, solar_dtype_t dt, const void* H, float* gpart,
-                             const GramPlan& plan, cudaStream_t st) {
-  return dt == SOLAR_BF16 ? launch_t<__nv_bfloat16>(B, N, d, H, gpart, plan, st)
-                          : launch_t<float>(B, N, d, H, gpart, plan, st);
+                             int* status, const GramPlan& plan, cudaStream_t st) {
+  return dt == SOLAR_BF16 ? launch_t<__nv_bfloat16>(B, N, d, H, gpart, status, plan, st)
+                          : launch_t<float>(B, N, d, H, gpart, status, plan, st);
 }
 
 }  // namespace solar

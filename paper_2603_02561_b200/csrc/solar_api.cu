@@ -68,8 +68,11 @@ solar_status_t solar_gram_partials(int B, int N, int d, solar_dtype_t dt, const 
   SOLAR_TRY(check_ptr(H));
   SOLAR_TRY(check_ws(workspace, workspace_bytes, factor_ws_bytes(B, N, d)));
   const GramPlan plan = gram_plan(B, N);
-  return from_cuda(launch_gram_simt(B, N, d, dt, H, static_cast<float*>(workspace), plan,
-                                    static_cast<cudaStream_t>(stream)));
+  float* gpart = static_cast<float*>(workspace);
+  int* status = reinterpret_cast<int*>(static_cast<char*>(workspace) + gram_status_offset(B, N, d));
+  const cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (gram_umma_supported(N, d, dt)) return from_cuda(launch_gram_umma(B, N, d, H, gpart, status, plan, st));
+  return from_cuda(launch_gram_simt(B, N, d, dt, H, gpart, status, plan, st));
 }
 
 solar_status_t solar_eig_from_partials_ex(int B, int N, int d, int r, solar_dtype_t dt, int route,
@@ -86,8 +89,10 @@ solar_status_t solar_eig_from_partials_ex(int B, int N, int d, int r, solar_dtyp
     return SOLAR_ERR_INVALID_ARG;
   SOLAR_TRY(check_ws(workspace, workspace_bytes, factor_ws_bytes(B, N, d)));
   const GramPlan plan = gram_plan(B, N);
-  return from_cuda(launch_eig(B, d, r, dt, route, static_cast<const float*>(workspace), plan.splits,
-                              S, V, info, route_taken, static_cast<cudaStream_t>(stream)));
+  const int* status =
+      reinterpret_cast<const int*>(static_cast<const char*>(workspace) + gram_status_offset(B, N, d));
+  return from_cuda(launch_eig(B, d, r, dt, route, static_cast<const float*>(workspace), status,
+                              plan.splits, S, V, info, route_taken, static_cast<cudaStream_t>(stream)));
 }
 
 solar_status_t solar_eig_from_partials(int B, int N, int d, int r, solar_dtype_t dt, float* S,
@@ -151,8 +156,12 @@ solar_status_t solar_attn_apply(int B, int M, int d, int r, solar_dtype_t dt, co
   SOLAR_TRY(check_ptr(C));
   SOLAR_TRY(check_ptr(O));
   SOLAR_TRY(check_ws(workspace, workspace_bytes, attn_ws_bytes(B, d, r)));
+  const cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (attn_umma_supported(d, dt))
+    return from_cuda(launch_attn_umma(B, M, d, r, C, flags, O, static_cast<const char*>(workspace),
+                                      attn_ws_layout(d, r), st));
   return from_cuda(launch_attn_simt(B, M, d, r, dt, C, flags, O, static_cast<const char*>(workspace),
-                                    attn_ws_layout(d, r), static_cast<cudaStream_t>(stream)));
+                                    attn_ws_layout(d, r), st));
 }
 
 solar_status_t solar_svd_attention_fwd(int B, int M, int N, int d, int r, solar_dtype_t dt,

@@ -46,29 +46,37 @@ inline GramPlan gram_plan(int B, int N) {
   return p;
 }
 
-// Workspace of the factorization: partial Grams [B][splits][d][d] fp32.
-inline size_t factor_ws_bytes(int B, int N, int d) {
+// Workspace of the factorization: partial Grams [B][splits][d][d] fp32, then one status
+// word per (user, slice), written by every Gram CTA: kGramStatusOk, or the code of the
+// bounded device-side wait that ran out.
+constexpr int kGramStatusOk = 0x600D;
+inline size_t gram_status_offset(int B, int N, int d) {
   const GramPlan p = gram_plan(B, N);
   return align_up((size_t)B * p.splits * d * d * sizeof(float), 256);
 }
+inline size_t factor_ws_bytes(int B, int N, int d) {
+  const GramPlan p = gram_plan(B, N);
+  return gram_status_offset(B, N, d) + align_up((size_t)B * p.splits * sizeof(int), 256);
+}
 
 // Workspace of the attention call, per user (all segments 256-byte aligned):
-//   Tf   [d][r] fp32   folded score operand  scale * W_Q Key_r^T
-//   Vr   [r][d] fp32   Value_r
-//   Thi  [r][d] bf16   high half of T^T  (tensor-core operand image)
-//   Tlo  [r][d] bf16   low half of T^T   (T^T - Thi)
-//   VrT  [d][r] bf16   Value_r^T         (tensor-core operand image)
+//   Tf   [d][r]      fp32  folded score operand  scale * W_Q Key_r^T
+//   Vr   [r][d]      fp32  Value_r
+//   Tpk  [2][64][d]  bf16  T^T split into a high and a low bf16 half (rows >= r are zero):
+//                          the score GEMM's B operand, K-major, for the tensor-core kernel
+//   Vpk  [2][d][64]  bf16  Value_r^T, high and low halves (columns >= r are zero):
+//                          the output GEMM's B operand, K-major
+constexpr int kTokenSlots = 64;     // r <= 64 factor tokens, zero padded in the packed operands
 struct AttnWs {
-  size_t tf_off, vr_off, thi_off, tlo_off, vrt_off, per_user;
+  size_t tf_off, vr_off, tpk_off, vpk_off, per_user;
 };
 inline AttnWs attn_ws_layout(int d, int r) {
   AttnWs w;
   size_t o = 0;
   w.tf_off = o;  o += align_up((size_t)d * r * 4, 256);
   w.vr_off = o;  o += align_up((size_t)d * r * 4, 256);
-  w.thi_off = o; o += align_up((size_t)d * r * 2, 256);
-  w.tlo_off = o; o += align_up((size_t)d * r * 2, 256);
-  w.vrt_off = o; o += align_up((size_t)d * r * 2, 256);
+  w.tpk_off = o; o += align_up((size_t)2 * kTokenSlots * d * 2, 256);
+  w.vpk_off = o; o += align_up((size_t)2 * d * kTokenSlots * 2, 256);
   w.per_user = o;
   return w;
 }
@@ -78,10 +86,13 @@ inline size_t attn_ws_bytes(int B, int d, int r) {
 
 // ---- launchers (one per kernel file) --------------------------------------
 cudaError_t launch_gram_simt(int B, int N, int d, solar_dtype_t dt, const void* H, float* gpart,
+                             int* status, const GramPlan& plan, cudaStream_t st);
+bool gram_umma_supported(int N, int d, solar_dtype_t dt);
+cudaError_t launch_gram_umma(int B, int N, int d, const void* H, float* gpart, int* status,
                              const GramPlan& plan, cudaStream_t st);
 cudaError_t launch_eig(int B, int d, int r, solar_dtype_t dt, int route, const float* gpart,
-                       int splits, float* S, float* V, int* info, int* route_taken,
-                       cudaStream_t st);
+                       const int* gram_status, int splits, float* S, float* V, int* info,
+                       int* route_taken, cudaStream_t st);
 int eig_subspace_dim(int d, int r);
 cudaError_t launch_project_us(int B, int N, int d, int r, solar_dtype_t dt, const void* H,
                               const float* V, void* US, cudaStream_t st);
@@ -91,6 +102,9 @@ cudaError_t launch_attn_prepare(int B, int d, int r, solar_dtype_t dt, const flo
 cudaError_t launch_attn_simt(int B, int M, int d, int r, solar_dtype_t dt, const void* C,
                              unsigned flags, void* O, const char* ws, const AttnWs& lay,
                              cudaStream_t st);
+bool attn_umma_supported(int d, solar_dtype_t dt);
+cudaError_t launch_attn_umma(int B, int M, int d, int r, const void* C, unsigned flags, void* O,
+                             const char* ws, const AttnWs& lay, cudaStream_t st);
 
 // ---- device helpers ----------------------------------------------------------
 template <typename T> __device__ __forceinline__ float to_f32(T x);

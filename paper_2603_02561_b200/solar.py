@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libsolar_b200.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA = range(5)
 F32, BF16 = 0, 1
 FLAG_NO_SOFTMAX = 1
-INFO_NOT_CONVERGED, INFO_NONFINITE, INFO_NOT_CERTIFIED = 1, 2, 4
+INFO_NOT_CONVERGED, INFO_NONFINITE, INFO_NOT_CERTIFIED, INFO_DEVICE_WAIT = 1, 2, 4, 8
 ROUTE_AUTO, ROUTE_SUBSPACE, ROUTE_FULL = 0, 1, 2
 
 _c_int, _c_size, _c_vp, _c_float, _c_uint = (ctypes.c_int, ctypes.c_size_t, ctypes.c_void_p,
