@@ -5,9 +5,16 @@ One "step" = one pass of the whole hot path over one batch of B users: streaming
 H, Jacobi eigensolve, factor-token projections, candidate attention.  Metric: candidates x
 sequence positions per second = B*M*N / step time.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3] [--in-flight S]
+                    [--impl ours|reference]
 
-Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs its own batch of B
+The timed region replays CUDA graphs of whole steps (no host work between kernels).  With
+--in-flight S > 1, S independent batches are in flight on S streams (each with its own
+workspace and factors), which is how a serving process overlaps one request's eigensolve
+(16 CTAs) with another's streaming passes; S = 1 gives the single-call latency.  Both
+figures are printed; `value` is the one at the S given (default 4).
+
+Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs its own batches of B
 users (users are independent: no data-path collective), timing is max over ranks.
 """
 from __future__ import annotations
@@ -30,6 +37,10 @@ from paper_2603_02561_b200 import workloads as wl  # noqa: E402
 
 L2_BYTES = 126 * 2 ** 20
 KERNELS_PER_STEP = 4          # gram, eigensolve, factor-token projections, attention
+FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # 148 SMs x 128 FMA lanes x 2 flop at 1965 MHz
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
+# profiles/ (null once the kernel has changed since the capture)
+TRAFFIC = {}
 
 
 def peaks():
@@ -157,13 +168,37 @@ def run_reference(args, w: wl.Workload):
 
 
 # ---------------------------------------------------------------------------------------
+def eig_flops(w: wl.Workload, iters: float, sweeps: float, route_full: bool) -> float:
+    """Useful floating-point operations of the eigensolver for one batch (both routes counted
+    from their loop bounds: dense products 2mnk, a 2x2 Jacobi block update 24 flop for the
+    matrix and 12 for the vectors)."""
+    d = w.d
+    if route_full:
+        return w.B * sweeps * (d - 1) * (d * d / 4) * 36.0
+    p = (w.r + 7) // 8 * 8
+    power = (iters + 1) * 2 * d * d * p + iters * (2 * d * p * p + p ** 3 / 3 + 2 * d * p * p) + 2 * d * p * p
+    jac = sweeps * (p - 1) * (p * p / 4) * 36.0
+    return w.B * (power + jac + 4 * d * p * p)
+
+
+class Lane:
+    """One in-flight slot: a stream with its own workspace and factor buffers."""
+
+    def __init__(self, torch, solar, w, tdt):
+        self.stream = torch.cuda.Stream()
+        self.S = torch.empty(w.B, w.r, device="cuda")
+        self.V = torch.empty(w.B, w.d, w.r, device="cuda")
+        self.ws = solar.alloc_workspace(w.B, w.M, w.N, w.d, w.r, tdt)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3")
+    ap.add_argument("--in-flight", type=int, default=4, help="independent batches in flight (streams)")
     ap.add_argument("--cpu-users", type=int, default=8, help="users in the cpu_baseline sample")
     ap.add_argument("--ref-users", type=int, default=2, help="users per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -171,6 +206,8 @@ def main():
     w = wl.CONFIGS[args.workload]
 
     if args.impl == "reference":
+        if args.steps == 2000:
+            args.steps = 3
         run_reference(args, w)
         return
 
@@ -198,82 +235,136 @@ def main():
     batches = []
     for i in range(nb):
         wi = w.with_(seed_index=w.seed_index + 1000 * (rank * nb + i + 1))
-        inp = wl.generate(wi)
-        batches.append(inp)
+        batches.append(wl.generate(wi))
     Wq, Wk, Wv = (torch.from_numpy(batches[0][k]).cuda().to(tdt) for k in ("Wq", "Wk", "Wv"))
     dH = [torch.from_numpy(b["H"]).cuda().to(tdt) for b in batches]
     dC = [torch.from_numpy(b["C"]).cuda().to(tdt) for b in batches]
     dO = [torch.empty_like(c) for c in dC]
-    S = torch.empty(w.B, w.r, device="cuda"); V = torch.empty(w.B, w.d, w.r, device="cuda")
-    ws = solar.alloc_workspace(w.B, w.M, w.N, w.d, w.r, tdt)
-    stream = torch.cuda.current_stream()
+    main_stream = torch.cuda.Stream()
+    n_lanes = max(1, args.in_flight)
+    lanes = [Lane(torch, solar, w, tdt) for _ in range(n_lanes)]
 
-    def step(i):
-        k = i % nb
-        solar.lowrank_factor(dH[k], w.r, S=S, V=V, workspace=ws, M=w.M, stream=stream)
-        solar.svd_attention_fwd(dC[k], S, V, Wq, Wk, Wv, w.scale, 0, O=dO[k], workspace=ws, N=w.N,
-                                stream=stream)
+    def step(k, lane, stream):
+        solar.lowrank_factor(dH[k], w.r, S=lane.S, V=lane.V, workspace=lane.ws, M=w.M, stream=stream)
+        solar.svd_attention_fwd(dC[k], lane.S, lane.V, Wq, Wk, Wv, w.scale, 0, O=dO[k], workspace=lane.ws,
+                                N=w.N, stream=stream)
+
+    def capture(n_steps, use_lanes):
+        """A CUDA graph of n_steps whole steps, dealt round-robin to the lanes' streams."""
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(main_stream):
+            with torch.cuda.graph(g, stream=main_stream, capture_error_mode="relaxed"):
+                if len(use_lanes) == 1:
+                    for i in range(n_steps):
+                        step(i % nb, use_lanes[0], main_stream)
+                else:
+                    fork = torch.cuda.Event()
+                    fork.record(main_stream)
+                    for li, lane in enumerate(use_lanes):
+                        lane.stream.wait_event(fork)
+                        for i in range(li, n_steps, len(use_lanes)):
+                            step(i % nb, lane, lane.stream)
+                        join = torch.cuda.Event()
+                        join.record(lane.stream)
+                        main_stream.wait_event(join)
+        return g
 
     def sync_all():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(max(args.warmup, 3)):
-        step(i)
+    def timed_replays(g, n):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(main_stream):
+            e0.record(main_stream)
+            for _ in range(n):
+                g.replay()
+            e1.record(main_stream)
+        return e0, e1
+
+    # the first call on a device sets kernel attributes: keep it outside any capture
+    for lane in lanes:
+        step(0, lane, main_stream)
+    torch.cuda.synchronize()
+
+    steps_per_graph = 4 * nb * n_lanes if n_lanes > 1 else nb
+    replays = max(1, -(-args.steps // steps_per_graph))
+    steps = replays * steps_per_graph
+    g_main = capture(steps_per_graph, lanes)
+    g_single = capture(nb, lanes[:1]) if n_lanes > 1 else g_main
+    warm = max(1, -(-max(args.warmup, 3) // steps_per_graph))
+    with torch.cuda.stream(main_stream):
+        for _ in range(warm):
+            g_main.replay()
+            g_single.replay()
     sync_all()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
     sync_all()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for i in range(args.steps):
-        step(i)
-    e1.record(stream)
+    e0, e1 = timed_replays(g_main, replays)
     sync_all()
     ms = e0.elapsed_time(e1)
+    # single-call latency: one step at a time on one stream
+    single_reps = max(3, min(replays * steps_per_graph // nb, 100))
+    s0, s1 = timed_replays(g_single, single_reps)
+    sync_all()
+    ms_single = s0.elapsed_time(s1) / (single_reps * nb)
 
-    # per-stage timing (same inputs, same launch configuration), CUDA events on the launch stream
+    # per-stage timing: each kernel alone, nb launches (rotating batches) per graph replay
+    lane0 = lanes[0]
     info = torch.zeros(w.B, dtype=torch.int32, device="cuda")
+    taken = torch.zeros(w.B, dtype=torch.int32, device="cuda")
     stages = {
-        "gram": lambda k: solar.gram_partials(dH[k], ws, stream=stream),
-        "eig": lambda k: solar.eig_from_partials(w.B, w.N, w.d, w.r, tdt, S, V, info, ws, stream=stream),
-        "attn_prepare": lambda k: solar.attn_prepare(S, V, Wq, Wk, Wv, w.scale, ws, stream=stream),
-        "attn_apply": lambda k: solar.attn_apply(dC[k], w.r, 0, dO[k], ws, stream=stream),
+        "gram": lambda k, st: solar.gram_partials(dH[k], lane0.ws, stream=st),
+        "eig": lambda k, st: solar.eig_from_partials_ex(w.B, w.N, w.d, w.r, tdt, solar.ROUTE_AUTO, lane0.S,
+                                                        lane0.V, info, taken, lane0.ws, stream=st),
+        "attn_prepare": lambda k, st: solar.attn_prepare(lane0.S, lane0.V, Wq, Wk, Wv, w.scale, lane0.ws, stream=st),
+        "attn_apply": lambda k, st: solar.attn_apply(dC[k], w.r, 0, dO[k], lane0.ws, stream=st),
     }
-    reps = max(10, min(args.steps, 50))
     stage_ms = {}
+    route_words = None
     for name in ("gram", "eig", "attn_prepare", "attn_apply"):
         fn = stages[name]
-        if name == "attn_prepare":        # restore valid factors after timing the eigensolver
-            solar.gram_partials(dH[0], ws, stream=stream)
-            solar.eig_from_partials(w.B, w.N, w.d, w.r, tdt, S, V, info, ws, stream=stream)
-        for k in range(3):
-            fn(k % nb)
+        with torch.cuda.stream(main_stream):
+            if name in ("eig", "attn_prepare"):    # valid inputs for the stage under test
+                solar.gram_partials(dH[0], lane0.ws, stream=main_stream)
+            if name == "attn_prepare":
+                stages["eig"](0, main_stream)
+            if name == "attn_apply":
+                solar.gram_partials(dH[0], lane0.ws, stream=main_stream)
+                stages["eig"](0, main_stream)
+                stages["attn_prepare"](0, main_stream)
         torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        for k in range(reps):
-            fn(k % nb)
-        b.record(stream)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(main_stream):
+            with torch.cuda.graph(g, stream=main_stream, capture_error_mode="relaxed"):
+                for k in range(nb):
+                    fn(k, main_stream)
+            for _ in range(3):
+                g.replay()
         torch.cuda.synchronize()
-        stage_ms[name] = a.elapsed_time(b) / reps
+        reps = 20
+        a, b = timed_replays(g, reps)
+        torch.cuda.synchronize()
+        stage_ms[name] = a.elapsed_time(b) / (reps * nb)
+        if name == "eig":
+            route_words = taken.cpu().numpy()
     clocks = sampler.stop() if rank == 0 else None
 
     # end to end through the public API with host buffers (pinned), copies inside the timed region
     hH = torch.from_numpy(batches[0]["H"]).to(tdt).pin_memory()
     hC = torch.from_numpy(batches[0]["C"]).to(tdt).pin_memory()
     hO = torch.empty_like(hC).pin_memory()
-    e2e_steps = max(3, min(args.steps, 20))
+    e2e_steps = max(3, min(steps, 50))
 
     def e2e_step():
-        dH[0].copy_(hH, non_blocking=True); dC[0].copy_(hC, non_blocking=True)
-        solar.lowrank_factor(dH[0], w.r, S=S, V=V, workspace=ws, M=w.M, stream=stream)
-        solar.svd_attention_fwd(dC[0], S, V, Wq, Wk, Wv, w.scale, 0, O=dO[0], workspace=ws, N=w.N,
-                                stream=stream)
-        hO.copy_(dO[0], non_blocking=True)
+        with torch.cuda.stream(main_stream):
+            dH[0].copy_(hH, non_blocking=True); dC[0].copy_(hC, non_blocking=True)
+            step(0, lane0, main_stream)
+            hO.copy_(dO[0], non_blocking=True)
 
     for _ in range(3):
         e2e_step()
@@ -284,40 +375,61 @@ def main():
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
 
-    tmax = torch.tensor([ms, e2e_s], dtype=torch.float64, device="cuda")
+    tmax = torch.tensor([ms, e2e_s, ms_single], dtype=torch.float64, device="cuda")
     if world > 1:
         dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-    ms, e2e_s = float(tmax[0]), float(tmax[1])
+    ms, e2e_s, ms_single = float(tmax[0]), float(tmax[1]), float(tmax[2])
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
     pk = peaks()
-    ms_step = ms / args.steps
+    ms_step = ms / steps
     value = world * w.pairs / (ms_step * 1e-3)
     roof_s = max(ab["total"] / (pk["hbm_gbs"] * 1e9), algorithmic_flops(w) / (pk["bf16_tflops"] * 1e12))
     dominant = max(stage_ms, key=stage_ms.get)
-    gram_gbs = ab["gram"] / (stage_ms["gram"] * 1e-3) / 1e9
     tot = sum(stage_ms.values())
+    routes = sorted(set(int(x) & 0xFF for x in route_words))
+    iters = float(np.mean([(int(x) >> 8) & 0xFF for x in route_words]))
+    sweeps = float(np.mean([(int(x) >> 16) & 0xFF for x in route_words]))
+    eflops = eig_flops(w, iters, sweeps, route_full=(routes == [2]))
+    per_kernel = {
+        "gram": {"bound": "hbm", "achieved": ab["gram"] / (stage_ms["gram"] * 1e-3) / 1e9, "peak": pk["hbm_gbs"],
+                 "unit": "GB/s"},
+        "attn_apply": {"bound": "hbm", "achieved": ab["attn"] / (stage_ms["attn_apply"] * 1e-3) / 1e9,
+                       "peak": pk["hbm_gbs"], "unit": "GB/s"},
+        "eig": {"bound": "alu", "achieved": eflops / (stage_ms["eig"] * 1e-3) / 1e12, "peak": FP32_ALU_TFLOPS,
+                "unit": "TFLOP/s", "note": "serial Jacobi rounds on B of 148 SMs: latency-bound, see DESIGN.md"},
+        "attn_prepare": {"bound": "alu", "achieved": 6.0 * w.B * w.r * w.d * w.d / (stage_ms["attn_prepare"] * 1e-3) / 1e12,
+                         "peak": FP32_ALU_TFLOPS, "unit": "TFLOP/s"},
+    }
+    for v in per_kernel.values():
+        v["frac"] = v["achieved"] / v["peak"]
+    traffic = TRAFFIC.get((w.name, dominant))
+    roof = dict(per_kernel[dominant], kernel=dominant, traffic=traffic, peak_source=pk["source"])
     line = {
         "metric": "svd_attention_fwd_candidates_x_positions_per_sec",
-        "value": value, "unit": "pairs/s", "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+        "value": value, "unit": "pairs/s", "n_gpus": world, "steps": steps,
+        "warmup": warm * steps_per_graph, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "N": w.N, "d": w.d, "r": w.r, "M": w.M,
-                   "storage": w.dtype, "users_per_gpu": w.B,
+                   "storage": w.dtype, "users_per_gpu": w.B, "in_flight": n_lanes,
+                   "launch": f"CUDA graphs of {steps_per_graph} steps, {replays} replays",
                    "l2": f"inputs rotate over {nb} distinct batches ({nb * ab['total'] / 2**20:.0f} MiB > 126 MiB L2)"},
+        "single_call": {"ms_per_step": ms_single, "value": world * w.pairs / (ms_single * 1e-3),
+                        "note": "one step at a time on one stream (in_flight = 1)"},
         "path_roofline": {"bound": "hbm", "algorithmic_bytes": ab["total"],
                           "algorithmic_flops": algorithmic_flops(w),
                           "roofline_pairs_per_s": w.pairs / roof_s, "frac": value / world / (w.pairs / roof_s),
+                          "frac_single_call": (w.pairs / (ms_single * 1e-3)) / (w.pairs / roof_s),
                           "peak_source": pk["source"]},
-        "roofline": {"kernel": "gram", "bound": "hbm", "achieved": gram_gbs, "peak": pk["hbm_gbs"],
-                     "unit": "GB/s", "frac": gram_gbs / pk["hbm_gbs"], "traffic": None,
-                     "peak_source": pk["source"]},
+        "roofline": roof,
+        "roofline_by_kernel": per_kernel,
         "stage_ms": stage_ms, "stage_share": {k: v / tot for k, v in stage_ms.items()},
         "dominant_stage": dominant,
-        "gpu_launches": KERNELS_PER_STEP * args.steps,
+        "eig_route": {"routes": routes, "power_steps": iters, "jacobi_sweeps": sweeps},
+        "gpu_launches": KERNELS_PER_STEP * steps,
         "clocks": clocks,
         "e2e": {"value": world * w.pairs * e2e_steps / e2e_s, "unit": "pairs/s",
                 "h2d_bytes_per_step": hH.numel() * hH.element_size() + hC.numel() * hC.element_size(),

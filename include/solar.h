@@ -150,7 +150,9 @@ solar_status_t solar_eig_from_partials(int B, int N, int d, int r, solar_dtype_t
 
 /* As above with the route chosen by the caller.  route_taken (device, [B] ints, or
  * NULL) receives per user: route used (1 subspace, 2 full; 0 = non-finite input)
- * | power steps << 8 | Jacobi sweeps << 16. */
+ * | power steps << 8 | Jacobi sweeps << 16 | reason << 24, where reason says why the
+ * range finder was not certified: 1 no gap at the cut, 2 residual too large for its
+ * gap, 4 a kept eigenvalue not positive, 8 sweep cap, 16 non-finite pivot. */
 solar_status_t solar_eig_from_partials_ex(int B, int N, int d, int r, solar_dtype_t dt, int route,
                                           float* S, float* V, int* info, int* route_taken,
                                           void* workspace, size_t workspace_bytes, void* stream);

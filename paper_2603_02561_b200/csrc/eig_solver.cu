@@ -218,7 +218,7 @@ __device__ __forceinline__ void mul_XtY(const float* __restrict__ X, const float
 // ONE warp.  Lane j owns row j of L and column j of Li.  Step k computes column k of L
 // (a dot of row j with row k) and row k of Li (a dot of row k of L with column j of Li):
 // both use the same broadcast row of L, so the inverse rides in the latency shadow of the
-// factorisation.  A numerically dependent column (pivot below 1e-10 of its original diagonal
+// factorisation.  A numerically dependent column (pivot below 1e-13 of its original diagonal
 // entry) is deflated: its column of L and row of Li are zero, so Q gets a zero column there.
 // Returns false (uniformly) only for a non-finite pivot.
 __device__ __forceinline__ bool cholesky_inverse_warp(double* __restrict__ A,
@@ -252,9 +252,11 @@ __device__ __forceinline__ bool cholesky_inverse_warp(double* __restrict__ A,
     const double piv = __shfl_sync(0xffffffffu, c, k);
     const double ref = dref[k];
     if (!(piv < 1e300)) return false;                    // NaN or overflow
-    // A column whose part orthogonal to the earlier ones is below 1e-5 of its length is
-    // rounding residue of a rank-deficient block: it is dropped (zero column of Q).
-    const double inv = (piv > 1e-10 * ref) ? rsqrt_f64(piv) : 0.0;
+    // A column whose part orthogonal to the earlier ones is below 3e-7 of its length is
+    // rounding residue (Y is fp32) of a rank-deficient block: it is dropped (zero column
+    // of Q).  Above that the direction may be noisy but Q stays orthonormal: the
+    // arithmetic here is double, and any orthonormal basis serves the Rayleigh-Ritz step.
+    const double inv = (piv > 1e-13 * ref) ? rsqrt_f64(piv) : 0.0;
     if (mine && j >= k) A[j * ld + k] = c * inv;
     if (mine) Li[k * ld + j] = (j <= k) ? (e0 + e1) * inv : 0.0;
     __syncwarp();
@@ -377,8 +379,14 @@ __device__ __forceinline__ void rank_descending(const float* lam, int* order, in
   }
 }
 
-// route_taken[b] = route | power steps << 8 | Jacobi sweeps << 16
+// route_taken[b] = route | power steps << 8 | Jacobi sweeps << 16 | kWhy* bits << 24
 constexpr int kRouteSubspace = 1, kRouteFull = 2;
+// Why the subspace route's result was not certified (0 = it was, or it was not tried):
+constexpr int kWhyCut = 1;          // the trace bound does not separate theta_r from the rest
+constexpr int kWhyResidual = 2;     // a residual is too large for its gap
+constexpr int kWhyNotPositive = 4;  // a kept Ritz value is not positive (rank(H) < r)
+constexpr int kWhySweepCap = 8;     // the Ritz Jacobi hit its sweep cap
+constexpr int kWhyCholesky = 16;    // non-finite pivot in the Cholesky-QR
 
 template <int D>
 __global__ void __launch_bounds__(EigCfg<D>::THREADS, 1)
@@ -397,6 +405,7 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
   __shared__ double s_trace;
   __shared__ int s_flags[4];
   __shared__ int s_sweeps;
+  __shared__ int s_why;     // why the subspace route was not accepted (kWhy* bits)
 
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
 
@@ -431,6 +440,7 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
     *reinterpret_cast<float4*>(Gc + (e / (D / 4)) * LD + (e % (D / 4)) * 4) = g;
   }
   if (tid < 4) s_flags[tid] = 0;
+  if (tid == 0) { s_why = 0; s_sweeps = 0; }
   // a Gram CTA whose bounded wait ran out leaves a code other than kGramStatusOk
   int lost = 0;
   for (int s = tid; s < splits; s += NT) lost |= (gram_status[b * splits + s] != kGramStatusOk);
@@ -503,7 +513,7 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
         if (tid == 0) s_flags[3] = pd ? 0 : 1;
       }
       __syncthreads();
-      if (s_flags[3]) { ok = false; break; }
+      if (s_flags[3]) { ok = false; if (tid == 0) s_why |= kWhyCholesky; break; }
       apply_Linv_t<D>(Yb, Li, Zb, p, LPD, tid, NT);
       __syncthreads();
       // next power step (kept in Yb), Rayleigh-Ritz matrix T = Z^T (G Z), block residual G Z - Z T
@@ -604,11 +614,14 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
         float gap = (tid == r - 1) ? cut : thi - theta[ordp[tid + 1]];
         if (tid > 0) gap = fminf(gap, theta[ordp[tid - 1]] - thi);
         const float resn = sqrtf(res2[tid]);
+        if (!(cut > 0.f)) atomicOr(&s_why, kWhyCut);
+        if (!(thi > 0.f)) atomicOr(&s_why, kWhyNotPositive);
+        if (!(resn <= fmaxf(tol.eps_vec * gap, tol.floor_rel * th1))) atomicOr(&s_why, kWhyResidual);
         good = (cut > 0.f) && (thi > 0.f) &&
                (resn <= fmaxf(tol.eps_vec * gap, tol.floor_rel * th1));
         if (!(resn == resn)) good = 0;
       }
-      if (s_sweeps < 0) good = 0;          // Jacobi sweep cap reached
+      if (s_sweeps < 0) { good = 0; if (tid == 0) s_why |= kWhySweepCap; }   // Jacobi sweep cap reached
       ok = __syncthreads_and(good);
       have_vectors = true;
     }
@@ -634,7 +647,7 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
         if (info) info[b] = ok ? 0 : SOLAR_INFO_NOT_CERTIFIED;
         if (route_taken) {
           const int sw = s_sweeps;
-          route_taken[b] = kRouteSubspace | (iters << 8) | ((sw < 0 ? kMaxSweeps : sw) << 16);
+          route_taken[b] = kRouteSubspace | (iters << 8) | ((sw < 0 ? kMaxSweeps : sw) << 16) | (s_why << 24);
         }
       }
       return;
@@ -735,7 +748,7 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
   }
   if (tid == 0) {
     if (info) info[b] = converged ? 0 : SOLAR_INFO_NOT_CONVERGED;
-    if (route_taken) route_taken[b] = kRouteFull | (sweeps_done << 16);
+    if (route_taken) route_taken[b] = kRouteFull | (sweeps_done << 16) | (s_why << 24);
   }
 }
 
