@@ -8,8 +8,9 @@
 // into a high and a low bf16 half so that both GEMMs keep ~16 mantissa bits, zero padded
 // to 64 token slots.
 //
-// One CTA per user.  Each weight matrix is staged once in shared memory with coalesced
-// 16-byte loads; the three small products then run out of shared memory with 4 outputs
+// Two CTAs per user: one computes Key_r^T and T (W_K, W_Q), the other Value_r (W_V).
+// Each weight matrix is staged once in shared memory with coalesced 16-byte loads, all at
+// the start of the CTA; the small products then run out of shared memory with 4 outputs
 // per thread.
 #include "solar_internal.cuh"
 
@@ -38,10 +39,11 @@ attn_prepare_kernel(const float* __restrict__ S, const float* __restrict__ V,
                     float scale, int r, char* __restrict__ ws, AttnWs lay) {
   extern __shared__ __align__(16) float sm[];
   const int rp = (r + 3) & ~3;          // token pitch: rows of VS / KrT are read 4 at a time
-  float* Ws = sm;                       // [D][D]   the weight matrix in use
-  float* VS = Ws + D * D;               // [D][rp]  V Sigma (zero in the padding)
+  float* Ws = sm;                       // [D][D]   W_K (role 0) or W_V (role 1)
+  float* Wq_s = Ws + D * D;             // [D][D]   W_Q (role 0)
+  float* VS = Wq_s + D * D;             // [D][rp]  V Sigma (zero in the padding)
   float* KrT = VS + D * rp;             // [D][rp]  Key_r^T
-  const int b = blockIdx.x, tid = threadIdx.x;
+  const int b = blockIdx.x, role = blockIdx.y, tid = threadIdx.x;
   char* wsb = ws + (size_t)b * lay.per_user;
   float* Tf = reinterpret_cast<float*>(wsb + lay.tf_off);
   float* Vr = reinterpret_cast<float*>(wsb + lay.vr_off);
@@ -49,19 +51,23 @@ attn_prepare_kernel(const float* __restrict__ S, const float* __restrict__ V,
   __nv_bfloat16* Vpk = reinterpret_cast<__nv_bfloat16*>(wsb + lay.vpk_off);
   const __nv_bfloat16 zero = __float2bfloat16_rn(0.f);
 
-  stage_weight<T, D>(Wk, Ws, tid);
+  stage_weight<T, D>(role == 0 ? Wk : Wv, Ws, tid);
+  if (role == 0) stage_weight<T, D>(Wq, Wq_s, tid);
   for (int e = tid; e < D * rp; e += kPrepThreads) {
     const int k = e / rp, i = e % rp;
     VS[e] = i < r ? V[((size_t)b * D + k) * r + i] * S[(size_t)b * r + i] : 0.f;
   }
   // zero padding of the packed operands: token slots r .. 63
-  for (int e = tid; e < 2 * (kTokenSlots - r) * D; e += kPrepThreads) {
-    const int h = e / ((kTokenSlots - r) * D), rem = e % ((kTokenSlots - r) * D);
-    Tpk[((size_t)h * kTokenSlots + r) * D + rem] = zero;
-  }
-  for (int e = tid; e < 2 * D * (kTokenSlots - r); e += kPrepThreads) {
-    const int row = e / (kTokenSlots - r), i = r + e % (kTokenSlots - r);
-    Vpk[(size_t)row * kTokenSlots + i] = zero;      // row runs over [2][D]
+  if (role == 0) {
+    for (int e = tid; e < 2 * (kTokenSlots - r) * D; e += kPrepThreads) {
+      const int h = e / ((kTokenSlots - r) * D), rem = e % ((kTokenSlots - r) * D);
+      Tpk[((size_t)h * kTokenSlots + r) * D + rem] = zero;
+    }
+  } else {
+    for (int e = tid; e < 2 * D * (kTokenSlots - r); e += kPrepThreads) {
+      const int row = e / (kTokenSlots - r), i = r + e % (kTokenSlots - r);
+      Vpk[(size_t)row * kTokenSlots + i] = zero;      // row runs over [2][D]
+    }
   }
   __syncthreads();
 
@@ -78,6 +84,26 @@ attn_prepare_kernel(const float* __restrict__ S, const float* __restrict__ V,
     }
   };
 
+  if (role == 1) {
+    // Value_r (fp32) and Value_r^T (packed bf16 halves)
+    for (int t = tid; t < (rp / 4) * D; t += kPrepThreads) {
+      const int j = t % D, i0 = (t / D) * 4;
+      float acc[4];
+      project(acc, i0, j);
+#pragma unroll
+      for (int m = 0; m < 4; ++m) {
+        const int i = i0 + m;
+        if (i < r) {
+          Vr[i * D + j] = acc[m];
+          const __nv_bfloat16 hi = __float2bfloat16_rn(acc[m]);
+          Vpk[(size_t)j * kTokenSlots + i] = hi;
+          Vpk[(size_t)(D + j) * kTokenSlots + i] = __float2bfloat16_rn(acc[m] - __bfloat162float(hi));
+        }
+      }
+    }
+    return;
+  }
+
   // Key_r^T
   for (int t = tid; t < (rp / 4) * D; t += kPrepThreads) {
     const int j = t % D, i0 = (t / D) * 4;
@@ -86,34 +112,13 @@ attn_prepare_kernel(const float* __restrict__ S, const float* __restrict__ V,
     *reinterpret_cast<float4*>(KrT + j * rp + i0) = make_float4(acc[0], acc[1], acc[2], acc[3]);
   }
   __syncthreads();
-  stage_weight<T, D>(Wv, Ws, tid);
-  __syncthreads();
-  // Value_r (fp32) and Value_r^T (packed bf16 halves)
-  for (int t = tid; t < (rp / 4) * D; t += kPrepThreads) {
-    const int j = t % D, i0 = (t / D) * 4;
-    float acc[4];
-    project(acc, i0, j);
-#pragma unroll
-    for (int m = 0; m < 4; ++m) {
-      const int i = i0 + m;
-      if (i < r) {
-        Vr[i * D + j] = acc[m];
-        const __nv_bfloat16 hi = __float2bfloat16_rn(acc[m]);
-        Vpk[(size_t)j * kTokenSlots + i] = hi;
-        Vpk[(size_t)(D + j) * kTokenSlots + i] = __float2bfloat16_rn(acc[m] - __bfloat162float(hi));
-      }
-    }
-  }
-  __syncthreads();
-  stage_weight<T, D>(Wq, Ws, tid);
-  __syncthreads();
   // T[k][i] = scale * sum_j Wq[k][j] Key_r[i][j], four tokens i per thread
   for (int t = tid; t < (rp / 4) * D; t += kPrepThreads) {
     const int i0 = (t % (rp / 4)) * 4, k = t / (rp / 4);
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 8
     for (int j = 0; j < D; ++j) {
-      const float w = Ws[k * D + j];
+      const float w = Wq_s[k * D + j];
       const float4 kr = *reinterpret_cast<const float4*>(KrT + j * rp + i0);
       acc[0] = fmaf(w, kr.x, acc[0]); acc[1] = fmaf(w, kr.y, acc[1]);
       acc[2] = fmaf(w, kr.z, acc[2]); acc[3] = fmaf(w, kr.w, acc[3]);
@@ -137,7 +142,7 @@ cudaError_t launch_t(int B, int d, int r, const float* S, const float* V, const 
                      const void* Wk, const void* Wv, float scale, char* ws, const AttnWs& lay,
                      cudaStream_t st) {
   const int rp = (r + 3) & ~3;
-  const size_t smem = (size_t)(d * d + 2 * d * rp) * sizeof(float);
+  const size_t smem = (size_t)(2 * d * d + 2 * d * rp) * sizeof(float);
   const T* q = static_cast<const T*>(Wq);
   const T* k = static_cast<const T*>(Wk);
   const T* v = static_cast<const T*>(Wv);
@@ -146,7 +151,7 @@ cudaError_t launch_t(int B, int d, int r, const float* S, const float* V, const 
     cudaError_t e = cudaFuncSetAttribute(attn_prepare_kernel<T, DD>,                            \
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
     if (e != cudaSuccess) return e;                                                             \
-    attn_prepare_kernel<T, DD><<<B, kPrepThreads, smem, st>>>(S, V, q, k, v, scale, r, ws, lay); \
+    attn_prepare_kernel<T, DD><<<dim3(B, 2), kPrepThreads, smem, st>>>(S, V, q, k, v, scale, r, ws, lay); \
   }
   switch (d) {
     case 32: SOLAR_PREP(32) break;

@@ -781,7 +781,7 @@ cudaError_t launch_eig(int B, int d, int r, solar_dtype_t dt, int route, const f
                        int* route_taken, cudaStream_t st) {
   EigTol tol;
   if (dt == SOLAR_BF16) {
-    tol.eps_vec = 1e-3f; tol.floor_rel = 256.f * kUnit; tol.sweep_stop = 1e-4f;
+    tol.eps_vec = 1e-3f; tol.floor_rel = 256.f * kUnit; tol.sweep_stop = 1e-3f;
   } else {
     tol.eps_vec = 1e-5f; tol.floor_rel = 32.f * kUnit; tol.sweep_stop = 1e-5f;
   }
