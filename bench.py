@@ -33,6 +33,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+from paper_2603_02561_b200 import bench_plan as bp  # noqa: E402
 from paper_2603_02561_b200 import workloads as wl  # noqa: E402
 
 L2_BYTES = 126 * 2 ** 20
@@ -40,7 +41,12 @@ KERNELS_PER_STEP = 4          # gram, eigensolve, factor-token projections, atte
 FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # 148 SMs x 128 FMA lanes x 2 flop at 1965 MHz
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (null once the kernel has changed since the capture)
-TRAFFIC = {}
+TRAFFIC = {
+    ("c3", "gram"): 20988160,        # profiles/gram_umma_c3.md
+    ("c3", "attn_apply"): 4762880,   # profiles/attn_umma_c3.md (O still in L2 when the kernel ends)
+    ("c3", "eig"): 2425600,          # profiles/eig_kernel_c3.md
+    ("c3", "attn_prepare"): 182784,  # profiles/attn_prepare_c3.md
+}
 
 
 def peaks():
@@ -231,11 +237,8 @@ def main():
     tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
     ab = algorithmic_bytes(w)
     # rotate over enough distinct batches that a step's inputs are never L2-resident
-    nb = max(2, -(-int(1.5 * L2_BYTES) // ab["total"]))
-    batches = []
-    for i in range(nb):
-        wi = w.with_(seed_index=w.seed_index + 1000 * (rank * nb + i + 1))
-        batches.append(wl.generate(wi))
+    nb = bp.batches_to_exceed_l2(ab["total"], L2_BYTES)
+    batches = [wl.generate(w.with_(seed_index=si)) for si in bp.rank_seed_indices(w.seed_index, rank, nb)]
     Wq, Wk, Wv = (torch.from_numpy(batches[0][k]).cuda().to(tdt) for k in ("Wq", "Wk", "Wv"))
     dH = [torch.from_numpy(b["H"]).cuda().to(tdt) for b in batches]
     dC = [torch.from_numpy(b["C"]).cuda().to(tdt) for b in batches]
@@ -288,9 +291,7 @@ def main():
         step(0, lane, main_stream)
     torch.cuda.synchronize()
 
-    steps_per_graph = 4 * nb * n_lanes if n_lanes > 1 else nb
-    replays = max(1, -(-args.steps // steps_per_graph))
-    steps = replays * steps_per_graph
+    steps_per_graph, replays, steps = bp.replay_plan(args.steps, nb, n_lanes)
     g_main = capture(steps_per_graph, lanes)
     g_single = capture(nb, lanes[:1]) if n_lanes > 1 else g_main
     warm = max(1, -(-max(args.warmup, 3) // steps_per_graph))
@@ -375,10 +376,7 @@ def main():
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
 
-    tmax = torch.tensor([ms, e2e_s, ms_single], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-    ms, e2e_s, ms_single = float(tmax[0]), float(tmax[1]), float(tmax[2])
+    ms, e2e_s, ms_single = bp.max_over_ranks([ms, e2e_s, ms_single], dist if world > 1 else None, "cuda")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -386,7 +384,7 @@ def main():
 
     pk = peaks()
     ms_step = ms / steps
-    value = world * w.pairs / (ms_step * 1e-3)
+    value = bp.aggregate_throughput(w.pairs, world, ms_step)
     roof_s = max(ab["total"] / (pk["hbm_gbs"] * 1e9), algorithmic_flops(w) / (pk["bf16_tflops"] * 1e12))
     dominant = max(stage_ms, key=stage_ms.get)
     tot = sum(stage_ms.values())
