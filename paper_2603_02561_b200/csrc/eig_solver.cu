@@ -56,9 +56,9 @@ template <int D> struct EigCfg {
   // floats of the full route: Gc, Gn, Vm, lam[D], order[D]
   static constexpr int FULL_FLOATS = 3 * D * LD + 2 * D;
   // floats of the subspace route: Ad, Li [PMAX][LPD], dref [PMAX] (double, first: 16-byte aligned),
-  // Zb, Yb, Xb [D][PMAX], Tc, Tn, Wm [PMAX][LP], theta, res2, ordp [PMAX], pad
+  // Zb, Yb, Xb [D][PMAX], Tc, Tn, Wm [PMAX][LP], Tb, Wb [2][PMAX*(PMAX+2)], theta, res2, ordp [PMAX], pad
   static constexpr int SUB_FLOATS = 2 * (2 * PMAX * LPD + PMAX) + 3 * D * PMAX + 3 * PMAX * LP +
-                                    3 * PMAX + 3;
+                                    4 * PMAX * (PMAX + 2) + 3 * PMAX + 3;
   // D = 128: the subspace buffers alias Gn and Vm (free until the full route starts)
   static constexpr bool ALIAS = (D == 128);
   static constexpr size_t SMEM =
@@ -307,39 +307,65 @@ __device__ __forceinline__ void rows_dot_col(const float* __restrict__ X, const 
 }
 
 // ---- Jacobi on the p x p Rayleigh-Ritz matrix ------------------------------------------
-// Run by the first jt = roundup((p/2)^2, 32) threads of the CTA (barrier id 1); thread
-// (I, J) of the (p/2) x (p/2) grid owns one 2x2 block per round.  T is double-buffered
-// in Tc/Tn ([p][lp]); W ([p][lp]) accumulates the rotations and must hold the identity
-// on entry.  flags[0..2] are sweep flags (zero on entry).  Returns the buffer that holds
-// the final matrix; *sweeps_out = sweeps used, negative if the cap was reached.
-__device__ __forceinline__ float* ritz_jacobi(float* Tc, float* Tn, float* W, int p, int lp,
-                                              float thr_abs2, float sweep_stop2,
-                                              volatile int* flags, int tid, int jt,
-                                              int* sweeps_out) {
+// Systolic form of the round-robin tournament: the matrix is indexed by SLOT, the pairs of
+// every round are the slots (2i, 2i+1), and after each round a fixed permutation moves the
+// slots (rows and columns of T, columns of W) so that in p-1 rounds every two indices meet
+// once.  Slot 0 stays; slot 1 -> 2; slot 2i -> 2i+2 (1 <= i <= p/2-2); slot p-2 -> p-1;
+// slot 2i+1 -> 2i-1 (i >= 1).  Nothing has to track which original index sits in a slot:
+// eigenvalue and eigenvector simply travel together.
+__device__ __forceinline__ int slot_next(int u, int p) {
+  if (u == 0) return 0;
+  if (u == 1) return 2;
+  if (u & 1) return u - 2;
+  return (u == p - 2) ? p - 1 : u + 2;
+}
+// Offset (in floats) of element (u, v) in the planar 2x2-block layout: block (u/2, v/2), whose
+// four entries sit in four planes [2*(u%2) + v%2][u/2][v/2] with row pitch p/2 + 1, so that
+// every scalar access of a warp (consecutive block columns, or the diagonal) is free of bank
+// conflicts -- both the reads of a thread's own block and the scattered writes of the moved one.
+__device__ __forceinline__ int blk_off(int u, int v, int hp) {
+  return (((u & 1) << 1) + (v & 1)) * (hp * (hp + 1)) + (u >> 1) * (hp + 1) + (v >> 1);
+}
+// Floats of one matrix in that layout.
+__device__ __forceinline__ int blk_size(int hp) { return 4 * hp * (hp + 1); }
+
+// Run by the first jt = roundup((p/2)^2, 32) threads of the CTA (barrier id 1).  Thread
+// (I, J) of the (p/2) x (p/2) grid owns block (I, J) of T and of W in every round: it reads
+// its block, the two diagonal blocks that define its row and column rotation, and its W
+// block, and writes the eight rotated entries to destinations fixed once per thread (the
+// slot move).  T and W are double-buffered ([2][blk_size] each; buffer 0 holds the input, W
+// the identity).  Returns the sweeps used (negative: cap reached); the result is in buffer
+// (sweeps*(p-1)) & 1.
+__device__ __forceinline__ int ritz_jacobi(float* Tb, float* Wb, int p, float thr_abs2,
+                                           float sweep_stop2, volatile int* flags, int tid, int jt) {
   const int hp = p >> 1;
+  const int plane = hp * (hp + 1), bufsz = 4 * plane;
   const bool active = tid < hp * hp;
   const int I = active ? tid / hp : 0, J = active ? tid % hp : 0;
-  float* w0 = W + 2 * I * lp;
-  float* w1 = w0 + lp;
+  const int src = I * (hp + 1) + J, srcI = I * (hp + 1) + I, srcJ = J * (hp + 1) + J;
+  const int r0 = slot_next(2 * I, p), r1 = slot_next(2 * I + 1, p);
+  const int c0 = slot_next(2 * J, p), c1 = slot_next(2 * J + 1, p);
+  const int t00 = blk_off(r0, c0, hp), t01 = blk_off(r0, c1, hp);
+  const int t10 = blk_off(r1, c0, hp), t11 = blk_off(r1, c1, hp);
+  const int w00 = blk_off(2 * I, c0, hp), w01 = blk_off(2 * I, c1, hp);   // W's rows stay put
+  const int w10 = blk_off(2 * I + 1, c0, hp), w11 = blk_off(2 * I + 1, c1, hp);
   int sweeps = -kMaxSweeps;
-  int ar, cr, ac, cc;
-  pair_start(I, p, ar, cr);
-  pair_start(J, p, ac, cc);
+  int cur = 0;
   for (int sweep = 0; sweep < kMaxSweeps; ++sweep) {
     if (tid == 0) flags[(sweep + 1) % 3] = 0;
     bool worst = false;
     for (int k = 0; k < p - 1; ++k) {
       if (active) {
-        const int pr = min(ar, cr), qr = max(ar, cr), pc = min(ac, cc), qc = max(ac, cc);
-        const float* tp = Tc + pr * lp;
-        const float* tq = Tc + qr * lp;
-        const float* up = Tc + pc * lp;
+        const float* Tc = Tb + cur * bufsz;
+        const float* Wc = Wb + cur * bufsz;
+        float* Tn = Tb + (cur ^ 1) * bufsz;
+        float* Wn = Wb + (cur ^ 1) * bufsz;
         bool big_r, big_c;
-        const Rot rr = jacobi_rot(tp[pr], tq[qr], tp[qr], thr_abs2, sweep_stop2, big_r);
-        const Rot rc = jacobi_rot(up[pc], Tc[qc * lp + qc], up[qc], thr_abs2, sweep_stop2, big_c);
+        const Rot rr = jacobi_rot(Tc[srcI], Tc[3 * plane + srcI], Tc[plane + srcI], thr_abs2, sweep_stop2, big_r);
+        const Rot rc = jacobi_rot(Tc[srcJ], Tc[3 * plane + srcJ], Tc[plane + srcJ], thr_abs2, sweep_stop2, big_c);
         worst |= big_c;
-        float x00 = tp[pc], x01 = tp[qc], x10 = tq[pc], x11 = tq[qc];
-        float w00 = w0[pc], w01 = w0[qc], w10 = w1[pc], w11 = w1[qc];
+        float x00 = Tc[src], x01 = Tc[plane + src], x10 = Tc[2 * plane + src], x11 = Tc[3 * plane + src];
+        float v00 = Wc[src], v01 = Wc[plane + src], v10 = Wc[2 * plane + src], v11 = Wc[3 * plane + src];
         if (I == J) {                      // the pair's own diagonal block
           const float tg = rc.t * x01;
           x00 -= tg; x11 += tg;
@@ -348,22 +374,17 @@ __device__ __forceinline__ float* ritz_jacobi(float* Tc, float* Tn, float* W, in
           rot_apply(rc, x00, x01); rot_apply(rc, x10, x11);   // columns
           rot_apply(rr, x00, x10); rot_apply(rr, x01, x11);   // rows
         }
-        rot_apply(rc, w00, w01); rot_apply(rc, w10, w11);
-        float* np_ = Tn + pr * lp;
-        float* nq_ = Tn + qr * lp;
-        np_[pc] = x00; np_[qc] = x01; nq_[pc] = x10; nq_[qc] = x11;
-        w0[pc] = w00; w0[qc] = w01; w1[pc] = w10; w1[qc] = w11;
-        pair_next(I, p, ar, cr);
-        pair_next(J, p, ac, cc);
+        rot_apply(rc, v00, v01); rot_apply(rc, v10, v11);
+        Tn[t00] = x00; Tn[t01] = x01; Tn[t10] = x10; Tn[t11] = x11;
+        Wn[w00] = v00; Wn[w01] = v01; Wn[w10] = v10; Wn[w11] = v11;
       }
       if (k == p - 2 && worst) flags[sweep % 3] = 1;
       bar_named(1, jt);
-      float* t = Tc; Tc = Tn; Tn = t;
+      cur ^= 1;
     }
     if (flags[sweep % 3] == 0) { sweeps = sweep + 1; break; }
   }
-  *sweeps_out = sweeps;
-  return Tc;
+  return sweeps;
 }
 
 // Ranks of lam[0..n) in descending order (ties: lower index first): order[rank] = index.
@@ -492,8 +513,10 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
     float* Xb = Yb + D * PM;                              // [D][p]    scratch / Ritz vectors
     float* Tc = Xb + D * PM;                              // [p][LP]
     float* Tn = Tc + PM * LP;
-    float* Wm = Tn + PM * LP;
-    float* theta = Wm + PM * LP;                          // [p]
+    float* Wm = Tn + PM * LP;                             // [p][LP]   Ritz eigenvectors, row-major
+    float* Tb = Wm + PM * LP;                             // [2][blk_size] Jacobi matrix, two buffers
+    float* Wb = Tb + 2 * PM * (PM + 2);                   // [2][blk_size] accumulated rotations
+    float* theta = Wb + 2 * PM * (PM + 2);                // [p]
     float* res2 = theta + PM;                             // [p]
     int* ordp = reinterpret_cast<int*>(res2 + PM);        // [p]
 
@@ -550,36 +573,32 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
     }
 
     if (ok) {
-      // symmetrise T, W = I
+      // symmetrise T into the planar block layout of the Jacobi, W = I
+      const int hp = p >> 1;
       for (int e = tid; e < p * p; e += NT) {
         const int a = e / p, c = e % p;
-        Wm[a * LP + c] = (a == c) ? 1.f : 0.f;
-        if (a < c) {
-          const float t = 0.5f * (Tc[a * LP + c] + Tc[c * LP + a]);
-          Tn[a * LP + c] = t; Tn[c * LP + a] = t;
-        } else if (a == c) {
-          Tn[a * LP + a] = Tc[a * LP + a];
-        }
+        Wb[blk_off(a, c, hp)] = (a == c) ? 1.f : 0.f;
+        Tb[blk_off(a, c, hp)] = 0.5f * (Tc[a * LP + c] + Tc[c * LP + a]);
       }
       __syncthreads();
       float tmax = 0.f;
-      for (int k = 0; k < p; ++k) tmax = fmaxf(tmax, fabsf(Tn[k * LP + k]));
-      const int hp = p >> 1;
+      for (int k = 0; k < p; ++k) tmax = fmaxf(tmax, fabsf(Tb[blk_off(k, k, hp)]));
       const int jt = min(NT, (hp * hp + 31) & ~31);
-      float* Tf = Tn;
       if (tid < jt) {
-        int sw;
-        Tf = ritz_jacobi(Tn, Tc, Wm, p, LP, (kTolAbs * tmax) * (kTolAbs * tmax), stop2, s_flags, tid, jt, &sw);
+        const int sw = ritz_jacobi(Tb, Wb, p, (kTolAbs * tmax) * (kTolAbs * tmax), stop2, s_flags, tid, jt);
         if (tid == 0) s_sweeps = sw;
       }
       __syncthreads();
-      // every thread needs the final buffer: the sweep count's parity decides it
+      // the result sits in the buffer given by the parity of the rounds done; unpack it
       {
         const int sw = s_sweeps;
-        const int rounds = (sw < 0 ? kMaxSweeps : sw) * (p - 1);
-        Tf = (rounds & 1) ? Tc : Tn;
+        const int fin = (((sw < 0 ? kMaxSweeps : sw) * (p - 1)) & 1) * blk_size(hp);
+        for (int e = tid; e < p * p; e += NT) {
+          const int a = e / p, c = e % p;
+          Wm[a * LP + c] = Wb[fin + blk_off(a, c, hp)];
+        }
+        if (tid < p) { theta[tid] = Tb[fin + blk_off(tid, tid, hp)]; res2[tid] = 0.f; }
       }
-      if (tid < p) { theta[tid] = Tf[tid * LP + tid]; res2[tid] = 0.f; }
       __syncthreads();
       rank_descending(theta, ordp, p, tid);
       __syncthreads();
