@@ -146,12 +146,13 @@ __device__ __forceinline__ float omega_entry(uint32_t e) {
   return sqrtf(-2.f * __logf(u1)) * __cosf(6.2831853f * u2);
 }
 
-// 1/sqrt(x) in double from the fp32 approximation and two Newton steps.
+// 1/sqrt(x) in double: the fp32 approximation (relative error 2^-22) and ONE Newton step
+// in double (2^-43).  That is ample for the Cholesky-QR -- a relative error e in a pivot's
+// inverse root scales one column of Q by 1 + e -- and every double-precision operation here
+// sits on the 32-step critical path of the factorisation.
 __device__ __forceinline__ double rsqrt_f64(double x) {
-  double y = (double)rsqrtf((float)x);
-  y = y * fma(-0.5 * x, y * y, 1.5);
-  y = y * fma(-0.5 * x, y * y, 1.5);
-  return y;
+  const double y = (double)rsqrtf((float)x);
+  return fma(y, fma(-0.5 * x * y, y, 0.5), y);
 }
 
 // ---- small dense products in shared memory -------------------------------------------
@@ -235,7 +236,21 @@ __device__ __forceinline__ bool cholesky_inverse_warp(double* __restrict__ A,
     double c0 = row[k], c1 = 0.0;
     double e0 = (j == k) ? 1.0 : 0.0, e1 = 0.0;
     int i = 0;
+    double c2 = 0.0, c3 = 0.0, e2 = 0.0, e3 = 0.0;
 #pragma unroll 2
+    for (; i + 3 < k; i += 4) {              // all ten loads of a 4-wide step are independent
+      const double2 lk0 = *reinterpret_cast<const double2*>(rk + i);
+      const double2 lk1 = *reinterpret_cast<const double2*>(rk + i + 2);
+      const double2 lj0 = *reinterpret_cast<const double2*>(row + i);
+      const double2 lj1 = *reinterpret_cast<const double2*>(row + i + 2);
+      const double x0 = Li[i * ld + j], x1 = Li[(i + 1) * ld + j];
+      const double x2 = Li[(i + 2) * ld + j], x3 = Li[(i + 3) * ld + j];
+      c0 = fma(-lj0.x, lk0.x, c0); c1 = fma(-lj0.y, lk0.y, c1);
+      c2 = fma(-lj1.x, lk1.x, c2); c3 = fma(-lj1.y, lk1.y, c3);
+      e0 = fma(-lk0.x, x0, e0);    e1 = fma(-lk0.y, x1, e1);
+      e2 = fma(-lk1.x, x2, e2);    e3 = fma(-lk1.y, x3, e3);
+    }
+    c0 += c2; c1 += c3; e0 += e2; e1 += e3;
     for (; i + 1 < k; i += 2) {
       const double2 lk = *reinterpret_cast<const double2*>(rk + i);
       const double2 lj = *reinterpret_cast<const double2*>(row + i);
@@ -432,39 +447,33 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
 
   // ---- G = sum of the slices' partial Grams, in slice order -----------------
   const float4* gp = reinterpret_cast<const float4*>(gpart + (size_t)b * splits * D * D);
-  int bad = 0;
-  for (int e = tid; e < D * D / 4; e += NT) {
-    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
-    int s = 0;
-    for (; s + 8 <= splits; s += 8) {          // eight independent loads in flight
-      float4 v[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) v[u] = __ldg(gp + (size_t)(s + u) * (D * D / 4) + e);
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        a0 += (double)v[u].x; a1 += (double)v[u].y; a2 += (double)v[u].z; a3 += (double)v[u].w;
-      }
-    }
-    if (s < splits) {                           // the remaining 1..7 slices, still loaded together
-      float4 v[7];
-#pragma unroll
-      for (int u = 0; u < 7; ++u)
-        v[u] = (s + u < splits) ? __ldg(gp + (size_t)(s + u) * (D * D / 4) + e)
-                                : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-      for (int u = 0; u < 7; ++u) {
-        a0 += (double)v[u].x; a1 += (double)v[u].y; a2 += (double)v[u].z; a3 += (double)v[u].w;
-      }
-    }
-    const float4 g = make_float4((float)a0, (float)a1, (float)a2, (float)a3);
-    bad |= !(isfinite(g.x) && isfinite(g.y) && isfinite(g.z) && isfinite(g.w));
-    *reinterpret_cast<float4*>(Gc + (e / (D / 4)) * LD + (e % (D / 4)) * 4) = g;
-  }
-  if (tid < 4) s_flags[tid] = 0;
-  if (tid == 0) { s_why = 0; s_sweeps = 0; }
   // a Gram CTA whose bounded wait ran out leaves a code other than kGramStatusOk
   int lost = 0;
   for (int s = tid; s < splits; s += NT) lost |= (gram_status[b * splits + s] != kGramStatusOk);
+  int bad = 0;
+  for (int e = tid; e < D * D / 4; e += NT) {
+    // fp32 sums in a fixed order (eight slices at a time, pairwise within the eight): the
+    // partials are fp32 to begin with, and one rounding per level is far below their own error
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < splits; s += 8) {
+      float4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        v[u] = (s + u < splits) ? __ldg(gp + (size_t)(s + u) * (D * D / 4) + e)
+                                : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int h = 4; h >= 1; h >>= 1)
+#pragma unroll
+        for (int u = 0; u < h; ++u) {
+          v[u].x += v[u + h].x; v[u].y += v[u + h].y; v[u].z += v[u + h].z; v[u].w += v[u + h].w;
+        }
+      acc.x += v[0].x; acc.y += v[0].y; acc.z += v[0].z; acc.w += v[0].w;
+    }
+    bad |= !(isfinite(acc.x) && isfinite(acc.y) && isfinite(acc.z) && isfinite(acc.w));
+    *reinterpret_cast<float4*>(Gc + (e / (D / 4)) * LD + (e % (D / 4)) * 4) = acc;
+  }
+  if (tid < 4) s_flags[tid] = 0;
+  if (tid == 0) { s_why = 0; s_sweeps = 0; }
   lost = __syncthreads_or(lost);
   bad = __syncthreads_or(bad);
   if (bad || lost) {
@@ -527,7 +536,20 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
     bool ok = true, have_vectors = false;
     mul_G<D, LD>(Gc, Zb, Yb, p, tid, NT);          // Y = G Omega
     __syncthreads();
-    for (int it = 0; it < kMaxSubspaceIters && ok; ++it) {
+    // Two attempts.  The power iteration stops when the block residual reaches the rounding
+    // floor; the certification below then looks at each vector against its own gap.  If
+    // only a residual is too large there, the second attempt takes the power iteration one
+    // step further (Yb still holds G Z) and solves the Rayleigh-Ritz problem again; anything
+    // else goes to the full route.  (Stopping earlier and retrying more often costs more than
+    // it saves: a retry repeats the Jacobi solve.)
+    for (int attempt = 0; attempt < 2; ++attempt) {
+    if (attempt == 1) {
+      ok = true;
+      if (tid == 0) { s_why = 0; s_flags[0] = 0; s_flags[1] = 0; s_flags[2] = 0; }
+      __syncthreads();
+    }
+    const float settle = tol.floor_rel;
+    for (int it = iters; it < kMaxSubspaceIters && ok; ++it) {
       // Cholesky-QR of the power step's Y = G Z:  A = Y^T Y = L L^T,  Z = Y L^-T
       mul_XtY<D, double, double>(Yb, Yb, Ad, p, LPD, tid, NT);
       __syncthreads();
@@ -566,7 +588,7 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
       __syncthreads();
       float tmax = 0.f;
       for (int k = 0; k < p; ++k) tmax = fmaxf(tmax, fabsf(Tc[k * LP + k]));
-      const bool settled = sqrtf(res2[0]) <= tol.floor_rel * tmax;
+      const bool settled = sqrtf(res2[0]) <= settle * tmax;
       __syncthreads();
       // with oversampling (p > r) the extra directions never settle: two steps are the rule
       if (settled || (p > r && it >= 1)) break;
@@ -644,6 +666,10 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
       ok = __syncthreads_and(good);
       have_vectors = true;
     }
+    // retry only when a residual alone stood in the way and a power step is left
+    if (ok || !have_vectors || s_why != kWhyResidual || iters >= kMaxSubspaceIters) break;
+    __syncthreads();
+    }   // attempts
 
     if (ok || (route == kRouteSubspace && have_vectors)) {
       // sign gauge and output
