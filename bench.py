@@ -12,7 +12,7 @@ The timed region replays CUDA graphs of whole steps (no host work between kernel
 --in-flight S > 1, S independent batches are in flight on S streams (each with its own
 workspace and factors), which is how a serving process overlaps one request's eigensolve
 (16 CTAs) with another's streaming passes; S = 1 gives the single-call latency.  Both
-figures are printed; `value` is the one at the S given (default 4).
+figures are printed; `value` is the one at the S given (default 16).
 
 Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs its own batches of B
 users (users are independent: no data-path collective), timing is max over ranks.
@@ -204,7 +204,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3")
-    ap.add_argument("--in-flight", type=int, default=4, help="independent batches in flight (streams)")
+    ap.add_argument("--in-flight", type=int, default=16, help="independent batches in flight (streams)")
     ap.add_argument("--cpu-users", type=int, default=8, help="users in the cpu_baseline sample")
     ap.add_argument("--ref-users", type=int, default=2, help="users per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -46,7 +46,9 @@ struct EigTol {
 
 template <int D> struct EigCfg {
   static constexpr int NP = D / 2;                 // pairs per round
-  static constexpr int PT = (D == 128) ? 2 : 1;    // row pairs (and column pairs) per thread
+  // row pairs (and column pairs) per thread: d = 64 runs on 256 threads so that the CTA
+  // leaves registers and shared memory for other kernels' CTAs on its SM
+  static constexpr int PT = (D == 32) ? 1 : 2;
   static constexpr int SIDE = NP / PT;             // threads along each side of the block grid
   static constexpr int THREADS = SIDE * SIDE;
   static constexpr int LD = D + 4;                 // rows stay 16-byte aligned
@@ -59,11 +61,14 @@ template <int D> struct EigCfg {
   // Zb, Yb, Xb [D][PMAX], Tc, Tn, Wm [PMAX][LP], Tb, Wb [2][PMAX*(PMAX+2)], theta, res2, ordp [PMAX], pad
   static constexpr int SUB_FLOATS = 2 * (2 * PMAX * LPD + PMAX) + 3 * D * PMAX + 3 * PMAX * LP +
                                     4 * PMAX * (PMAX + 2) + 3 * PMAX + 3;
-  // D = 128: the subspace buffers alias Gn and Vm (free until the full route starts)
+  // The [D][PMAX] buffers of the subspace route always alias Gn and Vm (free until the full
+  // route starts); for D = 128 so do all the others.
   static constexpr bool ALIAS = (D == 128);
+  static constexpr int DPM_FLOATS = 3 * D * PMAX;
   static constexpr size_t SMEM =
-      (size_t)(FULL_FLOATS + (ALIAS ? 0 : SUB_FLOATS)) * sizeof(float);
+      (size_t)(FULL_FLOATS + (ALIAS ? 0 : SUB_FLOATS - DPM_FLOATS)) * sizeof(float);
   static_assert(!ALIAS || SUB_FLOATS <= 2 * D * LD, "subspace buffers must fit in Gn+Vm");
+  static_assert(DPM_FLOATS <= 2 * D * LD && DPM_FLOATS % 4 == 0, "Zb, Yb, Xb must fit in Gn+Vm");
   static_assert((D * LD) % 4 == 0 && FULL_FLOATS % 4 == 0, "16-byte alignment of the regions");
 };
 
@@ -512,15 +517,15 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
   // ======================= route (1): certified subspace iteration =======================
   if (p > 0 && route != kRouteFull && gmax > 0.f) {
     constexpr int LP = Cfg::LP, PM = Cfg::PMAX;
-    float* sub = Cfg::ALIAS ? Gn : smem + Cfg::FULL_FLOATS;
+    float* sub = Cfg::ALIAS ? Gn + Cfg::DPM_FLOATS : smem + Cfg::FULL_FLOATS;
     constexpr int LPD = Cfg::LPD;
     double* Ad = reinterpret_cast<double*>(sub);          // [PM][LPD] Y^T Y, then its Cholesky factor
     double* Li = Ad + PM * LPD;                           // [PM][LPD] inverse of the factor
     double* dref = Li + PM * LPD;                         // [PM]      diagonal of Y^T Y
-    float* Zb = reinterpret_cast<float*>(dref + PM);      // [D][p]    orthonormal basis
+    float* Zb = Gn;                                       // [D][p]    orthonormal basis (over Gn, Vm)
     float* Yb = Zb + D * PM;                              // [D][p]    G Z
     float* Xb = Yb + D * PM;                              // [D][p]    scratch / Ritz vectors
-    float* Tc = Xb + D * PM;                              // [p][LP]
+    float* Tc = reinterpret_cast<float*>(dref + PM);      // [p][LP]
     float* Tn = Tc + PM * LP;
     float* Wm = Tn + PM * LP;                             // [p][LP]   Ritz eigenvectors, row-major
     float* Tb = Wm + PM * LP;                             // [2][blk_size] Jacobi matrix, two buffers
