@@ -208,8 +208,13 @@ def main():
     ap.add_argument("--cpu-users", type=int, default=8, help="users in the cpu_baseline sample")
     ap.add_argument("--ref-users", type=int, default=2, help="users per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="the c5 sweep: one JSON line per (N, r) point, with a brute-force softmax "
+                         "attention time on the host beside it")
+    ap.add_argument("--sweep-lengths", default="2048,4096,8192,16384,32768")
+    ap.add_argument("--sweep-ranks", default="8,16,32,64")
     args = ap.parse_args()
-    w = wl.CONFIGS[args.workload]
+    w = wl.lookup(args.workload)
 
     if args.impl == "reference":
         if args.steps == 2000:
@@ -234,6 +239,40 @@ def main():
         dist.barrier()
     solar.lib()
 
+    if args.sweep:
+        lengths = [int(x) for x in args.sweep_lengths.split(",")]
+        ranks = [int(x) for x in args.sweep_ranks.split(",")]
+        args.no_cpu_baseline = True
+        for wp in wl.sweep_configs(lengths=lengths, ranks=ranks):
+            line = measure(args, wp, torch, dist, solar, world, rank, local, light=True)
+            if rank == 0:
+                line["brute_force_cpu"] = brute_force_point(wp)
+                print(json.dumps(line), flush=True)
+            torch.cuda.empty_cache()
+    else:
+        line = measure(args, w, torch, dist, solar, world, rank, local)
+        if rank == 0:
+            print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def brute_force_point(w: wl.Workload) -> dict:
+    """Brute-force softmax attention over the N positions (Eq. 6-7, O(N M d)) of ONE user of
+    the point on the host cores, as candidates x positions per second."""
+    import oracle as o
+    Wq, Wk, Wv = wl.weights(w)
+    H = wl.history(w, 0).astype(np.float64)
+    C = wl.candidates(w, 0).astype(np.float64)
+    t0 = time.perf_counter()
+    o.softmax_attention(H, C, Wq, Wk, Wv, w.scale)
+    t = time.perf_counter() - t0
+    return {"value": w.M * w.N / t, "unit": "pairs/s", "seconds": t, "cores": cpu_threads(),
+            "sample": f"1 of {w.B} users, all {w.M} candidates", "kind": "oracle softmax_attention"}
+
+
+def measure(args, w, torch, dist, solar, world, rank, local, light=False):
+    """Times workload w on this rank's GPU; returns the JSON line (rank 0) or None."""
     tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
     ab = algorithmic_bytes(w)
     # rotate over enough distinct batches that a step's inputs are never L2-resident
@@ -359,7 +398,7 @@ def main():
     hH = torch.from_numpy(batches[0]["H"]).to(tdt).pin_memory()
     hC = torch.from_numpy(batches[0]["C"]).to(tdt).pin_memory()
     hO = torch.empty_like(hC).pin_memory()
-    e2e_steps = max(3, min(steps, 50))
+    e2e_steps = 3 if light else max(3, min(steps, 50))
 
     def e2e_step():
         with torch.cuda.stream(main_stream):
@@ -378,9 +417,7 @@ def main():
 
     ms, e2e_s, ms_single = bp.max_over_ranks([ms, e2e_s, ms_single], dist if world > 1 else None, "cuda")
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
+        return None
 
     pk = peaks()
     ms_step = ms / steps
@@ -439,9 +476,7 @@ def main():
         line["cpu_baseline"] = {"value": len(users) * w.M * w.N / t, "unit": "pairs/s",
                                 "cores": cpu_threads(), "kind": "oracle", "seconds": t,
                                 "sample": f"{len(users)} of {w.B} users, all {w.M} candidates"}
-    print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    return line
 
 
 if __name__ == "__main__":

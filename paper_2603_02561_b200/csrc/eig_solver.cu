@@ -17,13 +17,14 @@
 //  (2) Full route -- parallel two-sided Jacobi on the whole d x d matrix, always
 //      valid (Eq. 9's exact truncated SVD for any spectrum).
 //
-// Jacobi rounds use the round-robin tournament ordering (n/2 disjoint pairs per
-// round, n-1 rounds per sweep).  In one round every 2x2 block
-// G[{p,q}][{p',q'}] is touched by exactly one thread, which applies the row
-// pair's rotation from the left and the column pair's from the right.  Each
-// thread recomputes the (at most four) rotations it needs from the diagonal
-// blocks of the current matrix, and the matrix is double-buffered, so a round
-// costs ONE barrier.
+// Both Jacobi solves use the round-robin tournament in systolic form: the matrix is
+// indexed by slot, the pairs of every round are the slots (2i, 2i+1), and a fixed slot
+// move after each round makes every two indices meet once in n-1 rounds.  In one round
+// every 2x2 block is touched by exactly one thread, which applies the row pair's rotation
+// from the left and the column pair's from the right; each thread recomputes the
+// rotations it needs from the diagonal blocks of the current matrix, and the matrix is
+// double-buffered, so a round costs ONE barrier.  The 2x2 blocks are stored in four
+// planes so that every access of a warp is free of bank conflicts.
 #include <math.h>
 
 #include "solar_internal.cuh"
@@ -45,18 +46,16 @@ struct EigTol {
 };
 
 template <int D> struct EigCfg {
-  static constexpr int NP = D / 2;                 // pairs per round
-  // row pairs (and column pairs) per thread: d = 64 runs on 256 threads so that the CTA
-  // leaves registers and shared memory for other kernels' CTAs on its SM
-  static constexpr int PT = (D == 32) ? 1 : 2;
-  static constexpr int SIDE = NP / PT;             // threads along each side of the block grid
-  static constexpr int THREADS = SIDE * SIDE;
+  // d = 32 and d = 64 run on 256 threads (1 and 4 blocks per thread in the full route), so
+  // that a CTA leaves registers and shared memory for other kernels' CTAs on its SM;
+  // d = 128 needs 1024 (4 blocks per thread)
+  static constexpr int THREADS = (D == 128) ? 1024 : 256;
   static constexpr int LD = D + 4;                 // rows stay 16-byte aligned
   static constexpr int PMAX = (D >= 64) ? 32 : 16; // largest subspace dimension (<= D/2)
   static constexpr int LP = PMAX + 1;
   static constexpr int LPD = PMAX + 2;             // row pitch of the double matrices (16-byte rows)
-  // floats of the full route: Gc, Gn, Vm, lam[D], order[D]
-  static constexpr int FULL_FLOATS = 3 * D * LD + 2 * D;
+  // floats of the full route: Gc, Gn, Vm, lam[D], order[D], perm[2][D]
+  static constexpr int FULL_FLOATS = 3 * D * LD + 4 * D;
   // floats of the subspace route: Ad, Li [PMAX][LPD], dref [PMAX] (double, first: 16-byte aligned),
   // Zb, Yb, Xb [D][PMAX], Tc, Tn, Wm [PMAX][LP], Tb, Wb [2][PMAX*(PMAX+2)], theta, res2, ordp [PMAX], pad
   static constexpr int SUB_FLOATS = 2 * (2 * PMAX * LPD + PMAX) + 3 * D * PMAX + 3 * PMAX * LP +
@@ -110,18 +109,6 @@ __device__ __forceinline__ Rot jacobi_rot(float a, float b, float g, float thr_a
   r.t = act ? t : 0.f;
   r.tau = act ? s * y : 0.f;
   return r;
-}
-
-// Players (a, c) of pair i in the circle method on n players, advanced by one round:
-// pair 0 is (n-1, k); pair i > 0 is (k+i, k-i) modulo n-1.
-__device__ __forceinline__ void pair_start(int i, int n, int& a, int& c) {
-  a = (i == 0) ? n - 1 : i;
-  c = (i == 0) ? 0 : n - 1 - i;
-}
-__device__ __forceinline__ void pair_next(int i, int n, int& a, int& c) {
-  const int up_a = (a + 1 == n - 1) ? 0 : a + 1;
-  a = (i == 0) ? a : up_a;
-  c = (c + 1 == n - 1) ? 0 : c + 1;
 }
 
 __device__ __forceinline__ void rot_apply(const Rot& r, float& xp, float& xq) {
@@ -435,7 +422,7 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
            int p, int route, EigTol tol, float* __restrict__ S, float* __restrict__ V,
            int* __restrict__ info, int* __restrict__ route_taken) {
   using Cfg = EigCfg<D>;
-  constexpr int PT = Cfg::PT, SIDE = Cfg::SIDE, LD = Cfg::LD, NT = Cfg::THREADS;
+  constexpr int LD = Cfg::LD, NT = Cfg::THREADS;
   extern __shared__ __align__(16) float smem[];
   float* Gc = smem;                 // current matrix
   float* Gn = smem + D * LD;        // next matrix
@@ -706,99 +693,111 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
   }
 
   // ============================ route (2): full d x d Jacobi ============================
-  const int tI = tid / SIDE, tJ = tid % SIDE;
-  for (int e = tid; e < D * D; e += NT) {
-    const int i = e / D, j = e % D;
-    Vm[i * LD + j] = (i == j) ? 1.f : 0.f;
-  }
-  if (tid < 3) s_flags[tid] = 0;
-  __syncthreads();
-  int converged = 0, sweeps_done = kMaxSweeps;
-  int ar[PT], cr[PT], ac[PT], cc[PT];
-#pragma unroll
-  for (int a = 0; a < PT; ++a) {
-    pair_start(tI + a * SIDE, D, ar[a], cr[a]);
-    pair_start(tJ + a * SIDE, D, ac[a], cc[a]);
-  }
-  for (int sweep = 0; sweep < kMaxSweeps; ++sweep) {
-    if (tid == 0) s_flags[(sweep + 1) % 3] = 0;
-    bool worst = false;
-    for (int k = 0; k < D - 1; ++k) {
-      int pr[PT], qr[PT], pc[PT], qc[PT];
-      Rot rr[PT], rc[PT];
-#pragma unroll
-      for (int a = 0; a < PT; ++a) {
-        bool big_r, big_c;
-        pr[a] = min(ar[a], cr[a]); qr[a] = max(ar[a], cr[a]);
-        pc[a] = min(ac[a], cc[a]); qc[a] = max(ac[a], cc[a]);
-        rr[a] = jacobi_rot(Gc[pr[a] * LD + pr[a]], Gc[qr[a] * LD + qr[a]], Gc[pr[a] * LD + qr[a]],
-                           thr_abs2, stop2, big_r);
-        rc[a] = jacobi_rot(Gc[pc[a] * LD + pc[a]], Gc[qc[a] * LD + qc[a]], Gc[pc[a] * LD + qc[a]],
-                           thr_abs2, stop2, big_c);
-        worst |= big_c;
-      }
-#pragma unroll
-      for (int a = 0; a < PT; ++a) {
-        const float* gp_ = Gc + pr[a] * LD;
-        const float* gq_ = Gc + qr[a] * LD;
-        float* np_ = Gn + pr[a] * LD;
-        float* nq_ = Gn + qr[a] * LD;
-        float* v0 = Vm + 2 * (tI + a * SIDE) * LD;    // V' = V J_col on fixed rows (2I, 2I+1)
-        float* v1 = v0 + LD;
-#pragma unroll
-        for (int c = 0; c < PT; ++c) {
-          // G' = J_row^T G J_col on the block rows (p,q) x columns (p',q')
-          float x00 = gp_[pc[c]], x01 = gp_[qc[c]], x10 = gq_[pc[c]], x11 = gq_[qc[c]];
-          float v00 = v0[pc[c]], v01 = v0[qc[c]], v10 = v1[pc[c]], v11 = v1[qc[c]];
-          if (pr[a] == pc[c]) {            // the pair's own diagonal block
-            const float tg = rc[c].t * x01;
-            x00 -= tg; x11 += tg;
-            if (rc[c].s != 0.f) { x01 = 0.f; x10 = 0.f; }
-          } else {
-            rot_apply(rc[c], x00, x01); rot_apply(rc[c], x10, x11);   // columns
-            rot_apply(rr[a], x00, x10); rot_apply(rr[a], x01, x11);   // rows
-          }
-          rot_apply(rc[c], v00, v01); rot_apply(rc[c], v10, v11);
-          np_[pc[c]] = x00; np_[qc[c]] = x01; nq_[pc[c]] = x10; nq_[qc[c]] = x11;
-          v0[pc[c]] = v00; v0[qc[c]] = v01; v1[pc[c]] = v10; v1[qc[c]] = v11;
-        }
-      }
-#pragma unroll
-      for (int a = 0; a < PT; ++a) {
-        pair_next(tI + a * SIDE, D, ar[a], cr[a]);
-        pair_next(tJ + a * SIDE, D, ac[a], cc[a]);
-      }
-      if (k == D - 2 && worst) s_flags[sweep % 3] = 1;
-      __syncthreads();
-      float* t = Gc; Gc = Gn; Gn = t;
-    }
-    if (s_flags[sweep % 3] == 0) { converged = 1; sweeps_done = sweep + 1; break; }
-  }
+  // The same systolic slot form as the Ritz Jacobi, on the whole matrix.  T is kept in the
+  // planar block layout, double-buffered (buffer 0 overlays the row-major G, buffer 1 the
+  // next matrix slot); the eigenvector matrix W stays COLUMN-major and in place: slot v's
+  // vector is column perm[v], the slot move only permutes `perm`.  Lanes run along the row
+  // blocks I, so a warp reads one W column pair as 32 consecutive 8-byte pieces, the column
+  // rotation (and its perm lookup) is uniform across the warp, and every T access is
+  // conflict-free.  Thread (I, Jb) owns the blocks (I, Jb + c*NJ), c < PTJ.
+  {
+    constexpr int HP = D / 2, NJ = NT / HP, PTJ = HP / NJ, PLN = HP * (HP + 1), TBS = 4 * PLN;
+    static_assert(NT % HP == 0 && HP % NJ == 0 && TBS <= D * LD && D * D <= D * LD, "full-route tiling");
+    float* Wc = Vm;                                  // [D cols][D rows]
+    int* perm = order + D;                           // [2][D]
+    const int I = tid % HP, Jb = tid / HP;
 
-  // ---- order the eigenvalues, keep r, fix the sign of each vector ----------------
-  if (tid < D) lam[tid] = Gc[tid * LD + tid];
-  __syncthreads();
-  rank_descending(lam, order, D, tid);
-  __syncthreads();
-  float* sgn = Gn;   // reuse: [r] signs
-  if (tid < r) {
-    const int col = order[tid];
-    float best = -1.f, lead = 1.f;
-    for (int j = 0; j < D; ++j) {
-      const float v = Vm[j * LD + col];
-      if (fabsf(v) > best) { best = fabsf(v); lead = v; }   // strict: lowest index wins a tie
+    float xin[PTJ][4];
+#pragma unroll
+    for (int c = 0; c < PTJ; ++c) {
+      const int J = Jb + c * NJ;
+      xin[c][0] = Gc[(2 * I) * LD + 2 * J];     xin[c][1] = Gc[(2 * I) * LD + 2 * J + 1];
+      xin[c][2] = Gc[(2 * I + 1) * LD + 2 * J]; xin[c][3] = Gc[(2 * I + 1) * LD + 2 * J + 1];
     }
-    sgn[tid] = lead < 0.f ? -1.f : 1.f;
-    S[(size_t)b * r + tid] = sqrtf(fmaxf(lam[col], 0.f) / sc);
-  }
-  __syncthreads();
-  for (int e = tid; e < D * r; e += NT) {
-    const int j = e / r, i = e % r;
-    V[(size_t)b * D * r + e] = Vm[j * LD + order[i]] * sgn[i];
-  }
-  if (tid == 0) {
-    if (info) info[b] = converged ? 0 : SOLAR_INFO_NOT_CONVERGED;
-    if (route_taken) route_taken[b] = kRouteFull | (sweeps_done << 16) | (s_why << 24);
+    __syncthreads();                                 // all of row-major G is in registers
+    int tdst[PTJ][4];
+    const int r0 = slot_next(2 * I, D), r1 = slot_next(2 * I + 1, D);
+#pragma unroll
+    for (int c = 0; c < PTJ; ++c) {
+      const int J = Jb + c * NJ, src = I * (HP + 1) + J;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) Gc[q * PLN + src] = xin[c][q];
+      const int c0 = slot_next(2 * J, D), c1 = slot_next(2 * J + 1, D);
+      tdst[c][0] = blk_off(r0, c0, HP); tdst[c][1] = blk_off(r0, c1, HP);
+      tdst[c][2] = blk_off(r1, c0, HP); tdst[c][3] = blk_off(r1, c1, HP);
+    }
+    for (int e = tid; e < D * D; e += NT) Wc[e] = (e / D == e % D) ? 1.f : 0.f;
+    if (tid < D) perm[tid] = tid;
+    if (tid < 3) s_flags[tid] = 0;
+    __syncthreads();
+
+    const int srcI = I * (HP + 1) + I;
+    int converged = 0, sweeps_done = kMaxSweeps, cur = 0;
+    for (int sweep = 0; sweep < kMaxSweeps; ++sweep) {
+      if (tid == 0) s_flags[(sweep + 1) % 3] = 0;
+      bool worst = false;
+      for (int k = 0; k < D - 1; ++k) {
+        const float* Tc = cur ? Gn : Gc;
+        float* Tn = cur ? Gc : Gn;
+        const int* pc = perm + cur * D;
+        bool big_r, big_c;
+        const Rot rr = jacobi_rot(Tc[srcI], Tc[3 * PLN + srcI], Tc[PLN + srcI], thr_abs2, stop2, big_r);
+#pragma unroll
+        for (int c = 0; c < PTJ; ++c) {
+          const int J = Jb + c * NJ, srcJ = J * (HP + 1) + J, src = I * (HP + 1) + J;
+          const Rot rc = jacobi_rot(Tc[srcJ], Tc[3 * PLN + srcJ], Tc[PLN + srcJ], thr_abs2, stop2, big_c);
+          worst |= big_c;
+          float x00 = Tc[src], x01 = Tc[PLN + src], x10 = Tc[2 * PLN + src], x11 = Tc[3 * PLN + src];
+          float2* wa = reinterpret_cast<float2*>(Wc + pc[2 * J] * D + 2 * I);
+          float2* wb = reinterpret_cast<float2*>(Wc + pc[2 * J + 1] * D + 2 * I);
+          float2 va = *wa, vb = *wb;
+          if (I == J) {                      // the pair's own diagonal block
+            const float tg = rc.t * x01;
+            x00 -= tg; x11 += tg;
+            if (rc.s != 0.f) { x01 = 0.f; x10 = 0.f; }
+          } else {
+            rot_apply(rc, x00, x01); rot_apply(rc, x10, x11);   // columns
+            rot_apply(rr, x00, x10); rot_apply(rr, x01, x11);   // rows
+          }
+          rot_apply(rc, va.x, vb.x); rot_apply(rc, va.y, vb.y);
+          Tn[tdst[c][0]] = x00; Tn[tdst[c][1]] = x01; Tn[tdst[c][2]] = x10; Tn[tdst[c][3]] = x11;
+          *wa = va; *wb = vb;
+        }
+        if (tid < D) perm[(cur ^ 1) * D + slot_next(tid, D)] = pc[tid];
+        if (k == D - 2 && worst) s_flags[sweep % 3] = 1;
+        __syncthreads();
+        cur ^= 1;
+      }
+      if (s_flags[sweep % 3] == 0) { converged = 1; sweeps_done = sweep + 1; break; }
+    }
+
+    // ---- order the eigenvalues, keep r, fix the sign of each vector ----------------
+    const float* Tf = cur ? Gn : Gc;
+    const int* pf = perm + cur * D;
+    if (tid < D) lam[tid] = Tf[(tid & 1) * 3 * PLN + (tid >> 1) * (HP + 1) + (tid >> 1)];
+    __syncthreads();
+    rank_descending(lam, order, D, tid);
+    __syncthreads();
+    float* sgn = cur ? Gc : Gn;   // reuse: [r] signs
+    if (tid < r) {
+      const float* col = Wc + pf[order[tid]] * D;
+      float best = -1.f, lead = 1.f;
+      for (int j = 0; j < D; ++j) {
+        const float v = col[j];
+        if (fabsf(v) > best) { best = fabsf(v); lead = v; }   // strict: lowest index wins a tie
+      }
+      sgn[tid] = lead < 0.f ? -1.f : 1.f;
+      S[(size_t)b * r + tid] = sqrtf(fmaxf(lam[order[tid]], 0.f) / sc);
+    }
+    __syncthreads();
+    for (int e = tid; e < D * r; e += NT) {
+      const int j = e / r, i = e % r;
+      V[(size_t)b * D * r + e] = Wc[pf[order[i]] * D + j] * sgn[i];
+    }
+    if (tid == 0) {
+      if (info) info[b] = converged ? 0 : SOLAR_INFO_NOT_CONVERGED;
+      if (route_taken) route_taken[b] = kRouteFull | (sweeps_done << 16) | (s_why << 24);
+    }
   }
 }
 

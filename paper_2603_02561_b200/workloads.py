@@ -86,6 +86,16 @@ def sweep_configs(B=64, d=64, M=1024,
     return out
 
 
+def lookup(name: str) -> Workload:
+    """A named configuration: c1..c4, serve, or a point of the c5 sweep (c5_N<N>_r<r>)."""
+    if name in CONFIGS:
+        return CONFIGS[name]
+    for w in sweep_configs():
+        if w.name == name:
+            return w
+    raise KeyError(name)
+
+
 # --------------------------------------------------------------------------
 def _rng(seed: int, tensor: int, user: int) -> np.random.Generator:
     return np.random.Generator(np.random.Philox(key=[seed & (2**64 - 1), (tensor << 32) | user]))
