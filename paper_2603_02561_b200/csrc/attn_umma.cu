@@ -24,10 +24,11 @@ constexpr int kScoreCols = 64;             // tensor-memory columns reserved for
 template <int D> struct AttnCfg {
   static constexpr int KB = D / 64;                               // 64-wide K boxes of the score GEMM
   static constexpr int C_BYTES = KB * kBoxBytes;                  // candidate tile, reused for the output tile
-  static constexpr int T_BYTES = 2 * KB * kTokenSlots * 128;      // T^T hi/lo: [2][KB][64 rows][128 B]
+  // T^T hi/lo: [2][KB][np rows][128 B], np = 16 * ceil(r / 16) token rows (known at launch)
+  __host__ __device__ static constexpr int t_bytes(int np) { return 2 * KB * np * 128; }
   static constexpr int V_BYTES = 2 * D * 128;                     // Value_r^T hi/lo: [2][D rows][128 B]
   static constexpr int P_BYTES = 2 * kBoxBytes;                   // probabilities hi/lo
-  static constexpr size_t SMEM = (size_t)C_BYTES + T_BYTES + V_BYTES + P_BYTES + 1024;
+  static constexpr size_t smem(int np) { return (size_t)C_BYTES + t_bytes(np) + V_BYTES + P_BYTES + 1024; }
   static constexpr int TMEM_COLS = (D == 64) ? 128 : 256;         // scores (64) + output (D), power of two
 };
 
@@ -50,9 +51,7 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sC = base;                         // [KB][128 rows][128 B]
-  uint8_t* sT = sC + Cfg::C_BYTES;            // [2][KB][64 rows][128 B]
-  uint8_t* sV = sT + Cfg::T_BYTES;            // [2][D rows][128 B]
-  uint8_t* sP = sV + Cfg::V_BYTES;            // [2][128 rows][128 B]
+  uint8_t* sT = sC + Cfg::C_BYTES;            // [2][KB][np rows][128 B]
   __shared__ __align__(8) uint64_t bar_load, bar_s, bar_o;
   __shared__ uint32_t s_tmem;
   __shared__ int s_err;
@@ -60,6 +59,9 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
   const int b = blockIdx.y, m0 = blockIdx.x * kRows;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int np = (r + 15) & ~15;              // token slots the GEMMs run over (multiple of 16)
+  const int t_tile = np * 128;                // bytes of one [np rows][128 B] tile of T^T
+  uint8_t* sV = sT + Cfg::t_bytes(np);        // [2][D rows][128 B]   (a multiple of 2 KB further on)
+  uint8_t* sP = sV + Cfg::V_BYTES;            // [2][128 rows][128 B]
 
   if (tid == 0) {
     s_err = 0;
@@ -76,13 +78,13 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
   volatile int* err = &s_err;
 
   if (tid == 0) {
-    ptx::mbar_arrive_expect_tx(&bar_load, Cfg::C_BYTES + Cfg::T_BYTES + Cfg::V_BYTES);
+    ptx::mbar_arrive_expect_tx(&bar_load, Cfg::C_BYTES + Cfg::t_bytes(np) + Cfg::V_BYTES);
 #pragma unroll
     for (int x = 0; x < Cfg::KB; ++x) {
       ptx::tma_load_3d(sC + x * kBoxBytes, &tmC, &bar_load, x * 64, m0, b);
 #pragma unroll
       for (int h = 0; h < 2; ++h)     // rows h*64 .. h*64+63 of the packed T^T (hi, then lo)
-        ptx::tma_load_3d(sT + (h * Cfg::KB + x) * (kTokenSlots * 128), &tmT, &bar_load, x * 64,
+        ptx::tma_load_3d(sT + (h * Cfg::KB + x) * t_tile, &tmT, &bar_load, x * 64,
                          h * kTokenSlots, b);
     }
 #pragma unroll
@@ -101,7 +103,7 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t a = ptx::smem_u32(sC) + (kk / 4) * kBoxBytes + (kk % 4) * 32;
-          const uint32_t t = ptx::smem_u32(sT) + (h * Cfg::KB + kk / 4) * (kTokenSlots * 128) + (kk % 4) * 32;
+          const uint32_t t = ptx::smem_u32(sT) + (h * Cfg::KB + kk / 4) * t_tile + (kk % 4) * 32;
           ptx::umma_bf16_ss(tmem_s, ptx::umma_smem_desc(a, 0, 1024), ptx::umma_smem_desc(t, 0, 1024), idesc, acc);
           acc = true;
         }
@@ -239,16 +241,17 @@ cudaError_t launch_d(int B, int M, int r, const void* C, unsigned flags, void* O
   const uint64_t pu = lay.per_user;
   bool ok = encode_tmap_bf16_3d(&tmC, C, D, (uint64_t)M, (uint64_t)B, (uint64_t)D * 2, (uint64_t)M * D * 2, 64, kRows);
   ok = ok && encode_tmap_bf16_3d(&tmO, O, D, (uint64_t)M, (uint64_t)B, (uint64_t)D * 2, (uint64_t)M * D * 2, 64, kRows);
+  const int np = (r + 15) & ~15;
   ok = ok && encode_tmap_bf16_3d(&tmT, ws + lay.tpk_off, D, 2 * kTokenSlots, (uint64_t)B, (uint64_t)D * 2, pu, 64,
-                                 kTokenSlots);
+                                 np);
   ok = ok && encode_tmap_bf16_3d(&tmV, ws + lay.vpk_off, kTokenSlots, 2 * D, (uint64_t)B, kTokenSlots * 2, pu,
                                  kTokenSlots, D);
   if (!ok) return cudaErrorInvalidValue;
   cudaError_t e = cudaFuncSetAttribute(attn_umma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)Cfg::SMEM);
+                                       (int)Cfg::smem(kTokenSlots));
   if (e != cudaSuccess) return e;
   const dim3 grid((M + kRows - 1) / kRows, B), block(128);
-  attn_umma_kernel<D><<<grid, block, Cfg::SMEM, st>>>(tmC, tmO, tmT, tmV, r, flags,
+  attn_umma_kernel<D><<<grid, block, Cfg::smem(np), st>>>(tmC, tmO, tmT, tmV, r, flags,
                                                       static_cast<__nv_bfloat16*>(O), M);
   return cudaGetLastError();
 }
