@@ -53,6 +53,7 @@ attn_prepare_kernel(const float* __restrict__ S, const float* __restrict__ V,
 
   stage_weight<T, D>(role == 0 ? Wk : Wv, Ws, tid);
   if (role == 0) stage_weight<T, D>(Wq, Wq_s, tid);
+  pdl_wait();          // S and V come from the eigensolver; the workspace may still be in use before this
   for (int e = tid; e < D * rp; e += kPrepThreads) {
     const int k = e / rp, i = e % rp;
     VS[e] = i < r ? V[((size_t)b * D + k) * r + i] * S[(size_t)b * r + i] : 0.f;
@@ -70,6 +71,7 @@ attn_prepare_kernel(const float* __restrict__ S, const float* __restrict__ V,
     }
   }
   __syncthreads();
+  pdl_trigger();       // the next kernel may start launching while the products run
 
   // X[i][j] = sum_k VS[k][i] W[k][j] for four tokens i per thread; j runs along the lanes.
   auto project = [&](float (&acc)[4], int i0, int j) {
@@ -151,7 +153,9 @@ cudaError_t launch_t(int B, int d, int r, const float* S, const float* V, const 
     cudaError_t e = cudaFuncSetAttribute(attn_prepare_kernel<T, DD>,                            \
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
     if (e != cudaSuccess) return e;                                                             \
-    attn_prepare_kernel<T, DD><<<dim3(B, 2), kPrepThreads, smem, st>>>(S, V, q, k, v, scale, r, ws, lay); \
+    e = launch_pdl(attn_prepare_kernel<T, DD>, dim3(B, 2), dim3(kPrepThreads), smem, st, S, V, q, k, v, \
+                   scale, r, ws, lay);                                                           \
+    if (e != cudaSuccess) return e;                                                             \
   }
   switch (d) {
     case 32: SOLAR_PREP(32) break;

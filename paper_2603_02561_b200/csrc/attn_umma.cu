@@ -80,8 +80,10 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
   if (tid == 0) {
     ptx::mbar_arrive_expect_tx(&bar_load, Cfg::C_BYTES + Cfg::t_bytes(np) + Cfg::V_BYTES);
 #pragma unroll
+    for (int x = 0; x < Cfg::KB; ++x) ptx::tma_load_3d(sC + x * kBoxBytes, &tmC, &bar_load, x * 64, m0, b);
+    pdl_wait();        // the candidate tile is on its way; the packed operands come from the prepare kernel
+#pragma unroll
     for (int x = 0; x < Cfg::KB; ++x) {
-      ptx::tma_load_3d(sC + x * kBoxBytes, &tmC, &bar_load, x * 64, m0, b);
 #pragma unroll
       for (int h = 0; h < 2; ++h)     // rows h*64 .. h*64+63 of the packed T^T (hi, then lo)
         ptx::tma_load_3d(sT + (h * Cfg::KB + x) * t_tile, &tmT, &bar_load, x * 64,
@@ -114,6 +116,7 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
 
   // ---- softmax over the r tokens, one candidate row per thread -------------------------
   const bool have_s = ptx::mbar_wait(&bar_s, 0, err, kErrScores);
+  pdl_trigger();       // loads and the score GEMM are done: the next kernel may start launching
   __syncwarp();
   ptx::tc_fence_after_sync();
   const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
@@ -251,9 +254,8 @@ cudaError_t launch_d(int B, int M, int r, const void* C, unsigned flags, void* O
                                        (int)Cfg::smem(kTokenSlots));
   if (e != cudaSuccess) return e;
   const dim3 grid((M + kRows - 1) / kRows, B), block(128);
-  attn_umma_kernel<D><<<grid, block, Cfg::smem(np), st>>>(tmC, tmO, tmT, tmV, r, flags,
-                                                      static_cast<__nv_bfloat16*>(O), M);
-  return cudaGetLastError();
+  return launch_pdl(attn_umma_kernel<D>, grid, block, Cfg::smem(np), st, tmC, tmO, tmT, tmV, r, flags,
+                    static_cast<__nv_bfloat16*>(O), M);
 }
 
 }  // namespace

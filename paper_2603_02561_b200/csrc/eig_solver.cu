@@ -436,6 +436,7 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
   __shared__ int s_why;     // why the subspace route was not accepted (kWhy* bits)
 
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
+  pdl_wait();          // everything below reads what the Gram kernel wrote
 
   // ---- G = sum of the slices' partial Grams, in slice order -----------------
   const float4* gp = reinterpret_cast<const float4*>(gpart + (size_t)b * splits * D * D);
@@ -617,6 +618,7 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
       rank_descending(theta, ordp, p, tid);
       __syncthreads();
 
+      pdl_trigger();     // the long part is over: the next kernel may start launching
       // Ritz vectors v = Z w and residuals G v - theta v of the r kept pairs
       for (int t = tid; t < (D / 2) * p; t += NT) {
         const int jr = t % p, i0 = (t / p) * 2;
@@ -810,9 +812,8 @@ cudaError_t launch_d(int B, int r, int p, int route, EigTol tol, const float* gp
   cudaError_t e = cudaFuncSetAttribute(eig_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)Cfg::SMEM);
   if (e != cudaSuccess) return e;
-  eig_kernel<D><<<B, Cfg::THREADS, Cfg::SMEM, st>>>(gpart, gram_status, splits, r, p, route, tol, S,
-                                                    V, info, route_taken);
-  return cudaGetLastError();
+  return launch_pdl(eig_kernel<D>, dim3(B), dim3(Cfg::THREADS), Cfg::SMEM, st, gpart, gram_status, splits,
+                    r, p, route, tol, S, V, info, route_taken);
 }
 
 }  // namespace

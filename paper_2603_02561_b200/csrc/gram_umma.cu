@@ -102,9 +102,13 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tmap, float* __restrict__ g
 
   // ---- epilogue: tensor memory -> P[b,s] (row-major fp32) ------------------------------
   const bool done = ptx::mbar_wait(&accum_bar, 0, err, kErrEpilogue);
+  pdl_trigger();       // only the epilogue is left: the next kernel may start launching
   __syncwarp();
   ptx::tc_fence_after_sync();
   float* out = gpart + ((size_t)b * splits + s) * D * D;
+  // H has been streamed without waiting for the previous kernel on the stream (it may
+  // still be reading this workspace); nothing is written before it has completed.
+  pdl_wait();
   if (done && *err == 0) {
     // M = 128: accumulator row i sits in lane i.  M = 64: rows 16q .. 16q+15 sit in lanes
     // 32q .. 32q+15 (each warp reaches only its own 32-lane quarter).
@@ -142,9 +146,8 @@ cudaError_t launch_d(int B, int N, const void* H, float* gpart, int* status, con
                                        (int)Cfg::SMEM);   // per device, cheap next to the launch
   if (e != cudaSuccess) return e;
   const dim3 grid(plan.splits, B), block(128);
-  gram_umma_kernel<D><<<grid, block, Cfg::SMEM, st>>>(tmap, gpart, status, N, plan.chunk_tiles * kTileRows,
-                                                      plan.splits);
-  return cudaGetLastError();
+  return launch_pdl(gram_umma_kernel<D>, grid, block, Cfg::SMEM, st, tmap, gpart, status, N,
+                    plan.chunk_tiles * kTileRows, plan.splits);
 }
 
 }  // namespace

@@ -106,6 +106,29 @@ bool attn_umma_supported(int d, solar_dtype_t dt);
 cudaError_t launch_attn_umma(int B, int M, int d, int r, const void* C, unsigned flags, void* O,
                              const char* ws, const AttnWs& lay, cudaStream_t st);
 
+// ---- programmatic dependent launch ---------------------------------------------------
+// The four kernels of a forward pass run back to back on one stream.  Launched with this
+// attribute, a kernel may start while its predecessor is still draining; it does whatever
+// does not depend on the predecessor (barrier set-up, staging weights, streaming H or the
+// candidate tile) and then calls pdl_wait(), which returns once the predecessor has
+// completed and its writes are visible.  pdl_trigger() lets the successor start launching; it
+// is called late, when only a short tail is left, because CTAs that were launched early sit
+// on shared memory and registers while they wait and would crowd out concurrent streams.
+// Without the attribute both device calls are no-ops.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                              cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- device helpers ----------------------------------------------------------
 template <typename T> __device__ __forceinline__ float to_f32(T x);
 template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }
