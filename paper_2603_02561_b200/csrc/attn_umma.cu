@@ -37,6 +37,13 @@ __device__ __forceinline__ uint32_t swz(int row, int c) {
   return (uint32_t)row * 128u + (uint32_t)((c ^ (row & 7)) << 4);
 }
 
+// 2^x by the special-function unit (2 ulp; the probabilities are rounded to bf16 pairs anyway).
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&v);
@@ -144,7 +151,7 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
     float sum = 0.f;
 #pragma unroll
     for (int i = 0; i < kTokenSlots; ++i) {
-      p[i] = (i < r) ? exp2f((p[i] - mx) * 1.4426950408889634f) : 0.f;
+      p[i] = (i < r) ? fast_exp2((p[i] - mx) * 1.4426950408889634f) : 0.f;
       sum += p[i];
     }
     const float inv = 1.f / sum;
@@ -224,7 +231,7 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
 #pragma unroll
       for (int x = 0; x < Cfg::KB; ++x) ptx::tma_store_3d(&tmO, sC + x * kBoxBytes, x * 64, m0, b);
       ptx::tma_store_commit();
-      ptx::tma_store_wait_all();
+      ptx::tma_store_wait_read();
     }
   } else if (m0 + tid < M) {
     // a bounded wait ran out: the rows of this tile are marked NaN instead of left stale

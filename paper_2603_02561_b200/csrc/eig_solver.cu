@@ -57,9 +57,10 @@ template <int D> struct EigCfg {
   // floats of the full route: Gc, Gn, Vm, lam[D], order[D], perm[2][D]
   static constexpr int FULL_FLOATS = 3 * D * LD + 4 * D;
   // floats of the subspace route: Ad, Li [PMAX][LPD], dref [PMAX] (double, first: 16-byte aligned),
-  // Zb, Yb, Xb [D][PMAX], Tc, Tn, Wm [PMAX][LP], Tb, Wb [2][PMAX*(PMAX+2)], theta, res2, ordp [PMAX], pad
-  static constexpr int SUB_FLOATS = 2 * (2 * PMAX * LPD + PMAX) + 3 * D * PMAX + 3 * PMAX * LP +
-                                    4 * PMAX * (PMAX + 2) + 3 * PMAX + 3;
+  // Zb, Yb, Xb [D][PMAX], Tc, Wm [PMAX][LP], theta, res2, ordp [PMAX], pad; Tb, Wb [2][PMAX*(PMAX+2)] lie over Ad, Li
+  static constexpr int SUB_FLOATS = 2 * (2 * PMAX * LPD + PMAX) + 3 * D * PMAX + 2 * PMAX * LP +
+                                    3 * PMAX + 3;
+  static_assert(4 * PMAX * (PMAX + 2) <= 2 * (2 * PMAX * LPD + PMAX), "Tb, Wb must fit over Ad, Li, dref");
   // The [D][PMAX] buffers of the subspace route always alias Gn and Vm (free until the full
   // route starts); for D = 128 so do all the others.
   static constexpr bool ALIAS = (D == 128);
@@ -514,11 +515,12 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
     float* Yb = Zb + D * PM;                              // [D][p]    G Z
     float* Xb = Yb + D * PM;                              // [D][p]    scratch / Ritz vectors
     float* Tc = reinterpret_cast<float*>(dref + PM);      // [p][LP]
-    float* Tn = Tc + PM * LP;
-    float* Wm = Tn + PM * LP;                             // [p][LP]   Ritz eigenvectors, row-major
-    float* Tb = Wm + PM * LP;                             // [2][blk_size] Jacobi matrix, two buffers
+    float* Wm = Tc + PM * LP;                             // [p][LP]   Ritz eigenvectors, row-major
+    // The Jacobi's buffers lie over Ad, Li, dref: the Cholesky-QR is over when T is packed
+    // into them, and they are unpacked into Wm and theta before a retry orthonormalises again.
+    float* Tb = reinterpret_cast<float*>(Ad);             // [2][blk_size] Jacobi matrix, two buffers
     float* Wb = Tb + 2 * PM * (PM + 2);                   // [2][blk_size] accumulated rotations
-    float* theta = Wb + 2 * PM * (PM + 2);                // [p]
+    float* theta = Wm + PM * LP;                          // [p]
     float* res2 = theta + PM;                             // [p]
     int* ordp = reinterpret_cast<int*>(res2 + PM);        // [p]
 
