@@ -43,9 +43,9 @@ FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # 148 SMs x 128 FMA lanes x 2
 # profiles/ (null once the kernel has changed since the capture)
 TRAFFIC = {
     ("c3", "gram"): 20988160,        # profiles/gram_umma_c3.md
-    ("c3", "attn_apply"): 4762880,   # profiles/attn_umma_c3.md (O still in L2 when the kernel ends)
-    ("c3", "eig"): 2425600,          # profiles/eig_kernel_c3.md
-    ("c3", "attn_prepare"): 182784,  # profiles/attn_prepare_c3.md
+    ("c3", "attn_apply"): 4628224,   # profiles/attn_umma_c3.md (O still in L2 when the kernel ends)
+    ("c3", "eig"): 2430464,          # profiles/eig_kernel_c3.md
+    ("c3", "attn_prepare"): 183040,  # profiles/attn_prepare_c3.md
 }
 
 
