@@ -56,7 +56,7 @@ attn_prepare_kernel(const float* __restrict__ S, const float* __restrict__ V,
   pdl_wait();          // S and V come from the eigensolver; the workspace may still be in use before this
   for (int e = tid; e < D * rp; e += kPrepThreads) {
     const int k = e / rp, i = e % rp;
-    VS[e] = i < r ? V[((size_t)b * D + k) * r + i] * S[(size_t)b * r + i] : 0.f;
+    VS[e] = i < r ? V[((size_t)b * D + k) * r + i] * (S != nullptr ? S[(size_t)b * r + i] : 1.f) : 0.f;
   }
   // zero padding of the packed operands: token slots r .. 63
   if (role == 0) {

@@ -36,7 +36,7 @@ namespace {
 constexpr float kTolRel = 2.3841858e-07f;  // 2^-22: |g_pq| <= tol*sqrt(g_pp g_qq) counts as zero
 constexpr float kTolAbs = 7.4505806e-09f;  // 2^-27 of the largest diagonal entry
 constexpr float kUnit = 5.9604645e-08f;    // 2^-24, fp32 unit roundoff
-constexpr int kMaxSubspaceIters = 3;       // power steps before the subspace route gives up
+constexpr int kMaxSubspaceIters = 5;       // power steps before the subspace route gives up
 
 // Acceptance thresholds of the subspace route (chosen by the storage type).
 struct EigTol {

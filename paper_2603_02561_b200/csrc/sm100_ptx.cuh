@@ -126,14 +126,19 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 //     8-row groups; lbo is not used by the hardware for swizzled K-major layouts.
 //   MN-major operand (each K index is a 128-byte row of 64 MN elements): sbo = bytes between
 //     groups of 8 K indices, lbo = bytes between blocks of 64 MN elements.
-__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+// `layout` is the swizzle code of the descriptor: 2 = 128-byte, 4 = 64-byte, 6 = 32-byte rows.
+__device__ __forceinline__ uint64_t umma_smem_desc_sw(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes,
+                                                      uint32_t layout) {
   uint64_t d = 0;
   d |= static_cast<uint64_t>((saddr >> 4) & 0x3FFFu);
   d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
   d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
   d |= static_cast<uint64_t>(1) << 46;   // descriptor version of sm_100
-  d |= static_cast<uint64_t>(2) << 61;   // SWIZZLE_128B
+  d |= static_cast<uint64_t>(layout) << 61;
   return d;
+}
+__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return umma_smem_desc_sw(saddr, lbo_bytes, sbo_bytes, 2);   // SWIZZLE_128B
 }
 // Instruction descriptor of kind::f16 with bf16 operands and an fp32 accumulator.
 __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N, bool a_mn_major, bool b_mn_major) {
@@ -166,5 +171,10 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
 // outside the tensor.  Returns false when the driver entry point is missing or refuses.
 bool encode_tmap_bf16_3d(CUtensorMap* out, const void* base, uint64_t dim0, uint64_t dim1, uint64_t dim2,
                          uint64_t stride1_bytes, uint64_t stride2_bytes, uint32_t box0, uint32_t box1);
+// The same with the swizzle span chosen by the caller: 128, 64 or 32 bytes (the inner box must
+// be exactly that many bytes wide or narrower).
+bool encode_tmap_bf16_3d_sw(CUtensorMap* out, const void* base, uint64_t dim0, uint64_t dim1, uint64_t dim2,
+                            uint64_t stride1_bytes, uint64_t stride2_bytes, uint32_t box0, uint32_t box1,
+                            int swizzle_bytes);
 
 }  // namespace solar
