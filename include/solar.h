@@ -175,6 +175,32 @@ solar_status_t solar_attn_apply(int B, int M, int d, int r, solar_dtype_t dt, co
                                 void* workspace, size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------- *
+ * Softmax attention over the N history positions, evaluated through the factors:
+ *   O = softmax_rows( scale * (C W_Q W_K^T V) (U Sigma)^T ) (U Sigma) (V^T W_V)    [M,d]
+ * With H = U Sigma V^T of rank <= r this equals the softmax attention of Eq. 6-7,
+ * softmax(scale * Query Key^T) Value with Key = H W_K, Value = H W_V, at O(N M r)
+ * instead of O(N M d): the literal sense in which the factorization of Eq. 9 is
+ * lossless WITH the softmax.  It is not the paper's SVD-Attention operator (Eq. 12),
+ * which removes U (Eq. 10) and normalises over the r factor tokens; it is offered
+ * beside it because it needs nothing but the factors.
+ *
+ *   C        [B,M,d] dt (in)   candidate embeddings
+ *   US       [B,N,r] dt (in)   U Sigma = H V, as written by solar_lowrank_factor
+ *   V        [B,d,r] f32 (in)  right singular vectors (any sign convention: it cancels)
+ *   Wq,Wk,Wv [d,d] dt   (in)   shared by all users; y = x W
+ *   O        [B,M,d] dt (out)
+ *   workspace: solar_workspace_bytes() of the same sizes.
+ * One flash-attention style kernel per call (after the small per-user operand set-up):
+ * the N x M scores live in tensor memory only.  Supported: dt = SOLAR_BF16, d in
+ * {64, 128}, r in {16, 32, 64}; other shapes return SOLAR_ERR_UNSUPPORTED.
+ * ------------------------------------------------------------------------- */
+solar_status_t solar_factored_softmax_attention_fwd(int B, int M, int N, int d, int r, solar_dtype_t dt,
+                                                    const void* C, const void* US, const float* V,
+                                                    const void* Wq, const void* Wk, const void* Wv,
+                                                    float scale, void* O, void* workspace,
+                                                    size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------- *
  * Factorization without caller-provided scratch.  (The paper has no counterpart:
  * this is a packaging variant of solar_lowrank_factor, not another operation.)
  *

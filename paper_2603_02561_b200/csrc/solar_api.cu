@@ -186,4 +186,29 @@ solar_status_t solar_svd_attention_fwd(int B, int M, int N, int d, int r, solar_
   return solar_attn_apply(B, M, d, r, dt, C, flags, O, workspace, workspace_bytes, stream);
 }
 
+solar_status_t solar_factored_softmax_attention_fwd(int B, int M, int N, int d, int r, solar_dtype_t dt,
+                                                    const void* C, const void* US, const float* V,
+                                                    const void* Wq, const void* Wk, const void* Wv,
+                                                    float scale, void* O, void* workspace,
+                                                    size_t workspace_bytes, void* stream) {
+  SOLAR_TRY(check_dims(B, M, N, d, r, dt));
+  if (!flash_factored_supported(d, r, dt)) return SOLAR_ERR_UNSUPPORTED;
+  if (B == 0 || M == 0) return SOLAR_OK;
+  SOLAR_TRY(check_ptr(C));
+  SOLAR_TRY(check_ptr(US));
+  SOLAR_TRY(check_ptr(V));
+  SOLAR_TRY(check_ptr(Wq));
+  SOLAR_TRY(check_ptr(Wk));
+  SOLAR_TRY(check_ptr(Wv));
+  SOLAR_TRY(check_ptr(O));
+  SOLAR_TRY(check_ws(workspace, workspace_bytes, attn_ws_bytes(B, d, r)));
+  const cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const AttnWs lay = attn_ws_layout(d, r);
+  // The packed operands of the kernel are the prepare kernel's with unit singular values:
+  // T^T becomes (scale log2e W_Q W_K^T V)^T and Value_r^T becomes (V^T W_V)^T.
+  SOLAR_TRY(from_cuda(launch_attn_prepare(B, d, r, dt, nullptr, V, Wq, Wk, Wv,
+                                          scale * 1.4426950408889634f, static_cast<char*>(workspace), lay, st)));
+  return from_cuda(launch_flash_factored(B, M, N, d, r, C, US, O, static_cast<const char*>(workspace), lay, st));
+}
+
 }  // extern "C"

@@ -102,6 +102,9 @@ cudaError_t launch_attn_prepare(int B, int d, int r, solar_dtype_t dt, const flo
 cudaError_t launch_attn_simt(int B, int M, int d, int r, solar_dtype_t dt, const void* C,
                              unsigned flags, void* O, const char* ws, const AttnWs& lay,
                              cudaStream_t st);
+bool flash_factored_supported(int d, int r, solar_dtype_t dt);
+cudaError_t launch_flash_factored(int B, int M, int N, int d, int r, const void* C, const void* US, void* O,
+                                  const char* ws, const AttnWs& lay, cudaStream_t st);
 bool attn_umma_supported(int d, solar_dtype_t dt);
 cudaError_t launch_attn_umma(int B, int M, int d, int r, const void* C, unsigned flags, void* O,
                              const char* ws, const AttnWs& lay, cudaStream_t st);

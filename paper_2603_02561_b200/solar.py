@@ -37,6 +37,8 @@ SIGNATURES = {
                                    [_c_vp, _c_size, _c_vp]),
     "solar_project_us": (_c_int, [_c_int] * 4 + [_c_int] + [_c_vp] * 3 + [_c_vp]),
     "solar_attn_prepare": (_c_int, [_c_int] * 3 + [_c_int] + [_c_vp] * 5 + [_c_float, _c_vp, _c_size, _c_vp]),
+    "solar_factored_softmax_attention_fwd": (_c_int, [_c_int] * 5 + [_c_int] + [_c_vp] * 6 +
+                                             [_c_float, _c_vp, _c_vp, _c_size, _c_vp]),
     "solar_static_scratch_bytes": (_c_size, []),
     "solar_lowrank_factor_static": (_c_int, [_c_int] * 5 + [_c_int] + [_c_vp] * 4 + [_c_vp]),
     "solar_attn_apply": (_c_int, [_c_int] * 4 + [_c_int, _c_vp, _c_uint, _c_vp, _c_vp, _c_size, _c_vp]),
@@ -145,6 +147,26 @@ def svd_attention_fwd(C, S, V, Wq, Wk, Wv, scale, flags=0, O=None, workspace=Non
                                        int(flags), _ptr(O), _ptr(workspace), workspace.numel(),
                                        _stream(stream))
     _check(st, "solar_svd_attention_fwd")
+    return O
+
+
+def factored_softmax_attention_fwd(C, US, V, Wq, Wk, Wv, scale, O=None, workspace=None, stream=None):
+    """solar_factored_softmax_attention_fwd: softmax attention over the N positions through
+    the factors (US[B,N,r] = H V from lowrank_factor, V[B,d,r])."""
+    B, M, d = C.shape
+    N, r = US.shape[1], US.shape[2]
+    _need(C, (B, M, d), C.dtype, "C"); _need(US, (B, N, r), C.dtype, "US")
+    _need(V, (B, d, r), torch.float32, "V")
+    for nm, W in (("Wq", Wq), ("Wk", Wk), ("Wv", Wv)):
+        _need(W, (d, d), C.dtype, nm)
+    O = torch.empty_like(C) if O is None else O
+    _need(O, (B, M, d), C.dtype, "O")
+    if workspace is None:
+        workspace = alloc_workspace(B, M, N, d, r, C.dtype, C.device)
+    st = lib().solar_factored_softmax_attention_fwd(B, M, N, d, r, dtype_code(C.dtype), _ptr(C), _ptr(US),
+                                                    _ptr(V), _ptr(Wq), _ptr(Wk), _ptr(Wv), float(scale),
+                                                    _ptr(O), _ptr(workspace), workspace.numel(), _stream(stream))
+    _check(st, "solar_factored_softmax_attention_fwd")
     return O
 
 
