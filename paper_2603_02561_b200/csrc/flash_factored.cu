@@ -38,7 +38,10 @@ template <int D, int R> struct FlashCfg {
   static constexpr int Q_BYTES = 2 * kBox;            // Q' hi/lo, later y hi/lo: [2][128][128 B]
   static constexpr int P_BYTES = 2 * kBox;            // probabilities: [2 boxes of 64 positions][128][128 B]
   static constexpr int US_TILE = kPos * RB;           // one tile of U Sigma
-  static constexpr size_t SMEM = (size_t)C_BYTES + T_BYTES + V_BYTES + Q_BYTES + P_BYTES + 2 * US_TILE + 1024;
+  // the candidate tile (read once, by the Q' GEMM) and the output tile (written last) share
+  // the probabilities' buffer
+  static_assert(C_BYTES <= P_BYTES, "C and O tiles live in the P buffer");
+  static constexpr size_t SMEM = (size_t)T_BYTES + V_BYTES + Q_BYTES + P_BYTES + 2 * US_TILE + 1024;
   static constexpr int COL_Q = 0, COL_S = 64, COL_O = 192;      // tensor-memory columns
   static constexpr int TMEM_COLS = (D == 64) ? 256 : 512;
 };
@@ -91,18 +94,18 @@ __device__ __forceinline__ void tmem_row(uint32_t taddr, float (&x)[R]) {
 }
 
 template <int D, int R>
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(128, 2)
 flash_factored_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmO,
                       const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUtensorMap tmV,
                       const __grid_constant__ CUtensorMap tmUS, int N, int M, __nv_bfloat16* __restrict__ O) {
   using Cfg = FlashCfg<D, R>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sC = base;                         // [KB][128][128 B]
-  uint8_t* sT = sC + Cfg::C_BYTES;            // [2][KB][R][128 B]
+  uint8_t* sT = base;                         // [2][KB][R][128 B]
   uint8_t* sV = sT + Cfg::T_BYTES;            // [2][D][128 B]
   uint8_t* sQ = sV + Cfg::V_BYTES;            // [2][128][128 B]
   uint8_t* sP = sQ + Cfg::Q_BYTES;            // [2][128][128 B]
+  uint8_t* sC = sP;                           // [KB][128][128 B]  candidate tile first, output tile last
   uint8_t* sUS = sP + Cfg::P_BYTES;           // [2 stages][128][RB]
   __shared__ __align__(8) uint64_t bar_load, bar_q, bar_s, bar_y, bar_o, bar_us[2];
   __shared__ uint32_t s_tmem;
@@ -223,15 +226,19 @@ flash_factored_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_cons
 #pragma unroll
       for (int i = 0; i < 32; ++i) s[c * 32 + i] = __uint_as_float(v[i]);
     }
-    const int valid = min(kPos, N - t * kPos);      // positions past N hold zero-filled rows
+    const int valid = N - t * kPos;                 // positions past N hold zero-filled rows
+    if (valid < kPos) {
+#pragma unroll
+      for (int j = 0; j < kPos; ++j) s[j] = (j < valid) ? s[j] : -INFINITY;
+    }
     float m_new = m_run;
 #pragma unroll
-    for (int j = 0; j < kPos; ++j) m_new = (j < valid) ? fmaxf(m_new, s[j]) : m_new;
+    for (int j = 0; j < kPos; ++j) m_new = fmaxf(m_new, s[j]);
     const float alpha = ex2(m_run - m_new);         // 0 on the first tile (m_run = -inf)
     float sum = 0.f;
 #pragma unroll
     for (int j = 0; j < kPos; ++j) {
-      s[j] = (j < valid) ? ex2(s[j] - m_new) : 0.f;
+      s[j] = ex2(s[j] - m_new);                     // masked positions: 2^-inf = 0
       sum += s[j];
     }
     l_run = fmaf(l_run, alpha, sum);
