@@ -39,6 +39,7 @@ from paper_2603_02561_b200 import workloads as wl  # noqa: E402
 L2_BYTES = 126 * 2 ** 20
 KERNELS_PER_STEP = 4          # gram, eigensolve, factor-token projections, attention
 FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # 148 SMs x 128 FMA lanes x 2 flop at 1965 MHz
+SFU_TEXPS = 148 * 16 * 1.965e9 / 1e12              # 148 SMs x 16 special-function lanes at 1965 MHz
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (null once the kernel has changed since the capture)
 TRAFFIC = {
@@ -392,6 +393,35 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
         stage_ms[name] = a.elapsed_time(b) / (reps * nb)
         if name == "eig":
             route_words = taken.cpu().numpy()
+    # the factored-exact softmax attention over the N positions (beside the hot path, not part
+    # of `value`): factorization with U Sigma, then the flash-style kernel; timed alone
+    factored = None
+    if not light and w.dtype == "bf16" and w.d in (64, 128) and w.r in (16, 32, 64):
+        US = torch.empty(w.B, w.N, w.r, dtype=tdt, device="cuda")
+        with torch.cuda.stream(main_stream):
+            solar.lowrank_factor(dH[0], w.r, S=lane0.S, V=lane0.V, US=US, workspace=lane0.ws, M=w.M,
+                                 stream=main_stream)
+            for _ in range(2):
+                solar.factored_softmax_attention_fwd(dC[0], US, lane0.V, Wq, Wk, Wv, w.scale, O=dO[0],
+                                                     workspace=lane0.ws, stream=main_stream)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(main_stream):
+            with torch.cuda.graph(g, stream=main_stream, capture_error_mode="relaxed"):
+                for k in range(nb):
+                    solar.factored_softmax_attention_fwd(dC[k], US, lane0.V, Wq, Wk, Wv, w.scale, O=dO[k],
+                                                         workspace=lane0.ws, stream=main_stream)
+            g.replay()
+        torch.cuda.synchronize()
+        a, b = timed_replays(g, 5)
+        torch.cuda.synchronize()
+        f_ms = a.elapsed_time(b) / (5 * nb)
+        exps = float(w.pairs)
+        factored = {"ms_per_call": f_ms, "value": w.pairs / (f_ms * 1e-3), "unit": "pairs/s",
+                    "what": "solar_factored_softmax_attention_fwd (operand set-up + flash kernel), US resident",
+                    "roofline": {"bound": "alu", "achieved": exps / (f_ms * 1e-3) / 1e12, "peak": SFU_TEXPS,
+                                 "unit": "Texp/s", "frac": exps / (f_ms * 1e-3) / 1e12 / SFU_TEXPS,
+                                 "note": "one exp2 per candidate x position on the special-function units"}}
     clocks = sampler.stop() if rank == 0 else None
 
     # end to end through the public API with host buffers (pinned), copies inside the timed region
@@ -466,6 +496,7 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
         "eig_route": {"routes": routes, "power_steps": iters, "jacobi_sweeps": sweeps},
         "gpu_launches": KERNELS_PER_STEP * steps,
         "clocks": clocks,
+        "factored_exact": factored,
         "e2e": {"value": world * w.pairs * e2e_steps / e2e_s, "unit": "pairs/s",
                 "h2d_bytes_per_step": hH.numel() * hH.element_size() + hC.numel() * hC.element_size(),
                 "d2h_bytes_per_step": hO.numel() * hO.element_size(), "steps": e2e_steps},
