@@ -35,7 +35,7 @@ def _check(w, users_to_check, flags=0, want_us=False):
     return got, worst
 
 
-# ---- the BASELINE configurations ---------------------------------------------------
+# ---- the five named configurations ---------------------------------------------------
 def test_c1_fp32_exact_rank8():
     _check(wl.CONFIGS["c1"], [0])
 
