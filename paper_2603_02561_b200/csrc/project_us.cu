@@ -1,6 +1,7 @@
 // Optional left factor: US = U Sigma = H V  [B,N,r] in the storage type.
 // Eq. 10 eliminates U from the forward pass; this second pass over H serves
-// callers that want it (e.g. a backward pass through the SVD).
+// callers that want it (e.g. a backward pass through the SVD).  This file holds the FFMA
+// kernel for the shapes the tensor-core kernel does not take (fp32 storage, d = 32, N < 128).
 #include "solar_internal.cuh"
 
 namespace solar {
@@ -78,6 +79,7 @@ cudaError_t launch_t(int B, int N, int d, int r, const void* H, const float* V, 
 
 cudaError_t launch_project_us(int B, int N, int d, int r, solar_dtype_t dt, const void* H,
                               const float* V, void* US, cudaStream_t st) {
+  if (project_us_umma_supported(N, d, r, dt)) return launch_project_us_umma(B, N, d, r, H, V, US, st);
   return dt == SOLAR_BF16 ? launch_t<__nv_bfloat16>(B, N, d, r, H, V, US, st)
                           : launch_t<float>(B, N, d, r, H, V, US, st);
 }
