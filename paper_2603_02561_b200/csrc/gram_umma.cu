@@ -22,7 +22,9 @@ template <int D> struct GramCfg {
   static constexpr int BOXES = D / 64;                       // 64-column TMA boxes per tile
   static constexpr int BOX_BYTES = kTileRows * 128;          // 16 KB: 128 rows x 64 bf16
   static constexpr int TILE_BYTES = BOXES * BOX_BYTES;
-  static constexpr int STAGES = (D == 64) ? 6 : 4;
+  // Four 16/32 KB stages keep more than one SM's share of the HBM latency-bandwidth product in
+  // flight and leave room for two eigensolver CTAs (78 KB each at d = 64) beside a Gram CTA.
+  static constexpr int STAGES = 4;
   static constexpr size_t SMEM = (size_t)STAGES * TILE_BYTES + 1024;   // + slack to align to 1024
   static constexpr uint32_t IDESC = ptx::umma_idesc_bf16(D, D, true, true);
 };
