@@ -175,6 +175,30 @@ solar_status_t solar_attn_apply(int B, int M, int d, int r, solar_dtype_t dt, co
                                 void* workspace, size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------- *
+ * Backward pass of the truncated SVD with U absent from the forward pass (Eq. 13-15
+ * and the appendix that derives them):
+ *   dH = U [ diag(dS) + 2 Sigma sym(F o (dV^T V)) ] V^T,   U = H V Sigma^-1,
+ *   F_ij = D_ij / (D_ij^2 + eps^2),  D_ij = sigma_i^2 - sigma_j^2,  eps = eps_rel * sigma_max^2
+ * (eps_rel = 0 is Eq. 14 itself, with F_ij = 0 where D_ij = 0).  The Hadamard factor is
+ * dV^T V, the index order for which the formula is the derivative of the forward pass
+ * (the appendix's expansion of the trace has the indices transposed, which flips the sign
+ * of that term).  Evaluated as one more streaming pass over H:  dH_b = H_b K_b with
+ * K_b = V Sigma^-1 [.] V^T, so U is never materialised.
+ *
+ *   H   [B,N,d] dt  (in)   the histories given to solar_lowrank_factor
+ *   S   [B,r]  f32  (in)   singular values,  V [B,d,r] f32 (in) right singular vectors
+ *   dS  [B,r]  f32  (in)   dL/dSigma,        dV [B,d,r] f32 (in) dL/dV
+ *   dH  [B,N,d] dt  (out)  dL/dH; a direction with sigma_i = 0 contributes nothing
+ *   workspace: at least B*d*d*4 bytes (solar_workspace_bytes() of the same sizes is enough);
+ *   holds K_b [B,d,d] f32 on return.
+ * Two launches on `stream`; no synchronisation; nothing is allocated.
+ * ------------------------------------------------------------------------- */
+solar_status_t solar_svd_backward(int B, int N, int d, int r, solar_dtype_t dt, const void* H,
+                                  const float* S, const float* V, const float* dS, const float* dV,
+                                  float eps_rel, void* dH, void* workspace, size_t workspace_bytes,
+                                  void* stream);
+
+/* ------------------------------------------------------------------------- *
  * Softmax attention over the N history positions, evaluated through the factors:
  *   O = softmax_rows( scale * (C W_Q W_K^T V) (U Sigma)^T ) (U Sigma) (V^T W_V)    [M,d]
  * With H = U Sigma V^T of rank <= r this equals the softmax attention of Eq. 6-7,

@@ -1,7 +1,8 @@
-// Optional left factor: US = U Sigma = H V  [B,N,r] in the storage type.
-// Eq. 10 eliminates U from the forward pass; this second pass over H serves
-// callers that want it (e.g. a backward pass through the SVD).  This file holds the FFMA
-// kernel for the shapes the tensor-core kernel does not take (fp32 storage, d = 32, N < 128).
+// Right-multiplication of every history by a per-user matrix, Out_b = H_b X_b with X_b
+// [d][q] fp32 and Out [B,N,q] in the storage type: the optional left factor
+// US = U Sigma = H V (q = r; Eq. 10 eliminates U from the forward pass) and the backward
+// pass of the SVD, dH = H K (q = d; Eq. 15).  This file holds the FFMA kernel for the shapes
+// the tensor-core kernel does not take (fp32 storage, d = 32, N < 128).
 #include "solar_internal.cuh"
 
 namespace solar {
@@ -20,9 +21,10 @@ project_us_kernel(const T* __restrict__ H, const float* __restrict__ V, T* __res
   float* Vs = sm;                  // [D][kRP], zero padded
   float* Hs = sm + D * kRP;        // [kRows][D]
   const int b = blockIdx.y, n0 = blockIdx.x * kRows;
+  const int c0 = blockIdx.z * kRP;       // this CTA's 64 output columns
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (int e = tid; e < D * kRP; e += kWarps * 32) {
-    const int k = e / kRP, i = e % kRP;
+    const int k = e / kRP, i = c0 + e % kRP;
     Vs[e] = i < r ? V[((size_t)b * D + k) * r + i] : 0.f;
   }
   constexpr int VE = Vec16<T>::kElems;
@@ -45,16 +47,16 @@ project_us_kernel(const T* __restrict__ H, const float* __restrict__ V, T* __res
       s0 = fmaf(h[k], Vs[k * kRP + lane], s0);
       s1 = fmaf(h[k], Vs[k * kRP + lane + 32], s1);
     }
-    T* o = US + ((size_t)b * N + n0 + rr) * r;
-    if (lane < r) o[lane] = from_f32<T>(s0);
-    if (lane + 32 < r) o[lane + 32] = from_f32<T>(s1);
+    T* o = US + ((size_t)b * N + n0 + rr) * r + c0;
+    if (c0 + lane < r) o[lane] = from_f32<T>(s0);
+    if (c0 + lane + 32 < r) o[lane + 32] = from_f32<T>(s1);
   }
 }
 
 template <typename T>
 cudaError_t launch_t(int B, int N, int d, int r, const void* H, const float* V, void* US,
                      cudaStream_t st) {
-  const dim3 grid((N + kRows - 1) / kRows, B), block(kWarps * 32);
+  const dim3 grid((N + kRows - 1) / kRows, B, (r + kRP - 1) / kRP), block(kWarps * 32);
   const size_t smem = (size_t)(d * kRP + kRows * d) * sizeof(float);
   const T* h = static_cast<const T*>(H);
   T* u = static_cast<T*>(US);

@@ -1,13 +1,14 @@
-// Optional left factor on the tensor cores (bf16 storage, d = 64 or 128):
-//   US = U Sigma = H V   [B,N,r]
-// Eq. 10 eliminates U from the forward pass; this second streaming pass over H serves
-// callers that want it (attention over the N positions through the factors, a backward
-// pass through the SVD).
+// Right-multiplication of every history by a per-user matrix on the tensor cores (bf16
+// storage, d = 64 or 128):   Out_b = H_b X_b,   X_b [d][q] fp32,  q <= 128.
+// Two callers: the optional left factor  US = U Sigma = H V  (q = r; Eq. 10 eliminates U
+// from the forward pass, this second streaming pass over H serves attention over the N
+// positions through the factors) and the backward pass of the SVD, dH = H K (q = d; Eq. 15
+// with U = H V Sigma^-1).
 //
 // One CTA per (user, row slice), the same slicing as the Gram pass.  Warp 4 streams the
 // slice's 128-row tiles of H through a ring of shared-memory stages with TMA; warp 5
 // issues tcgen05.mma with the tile as the K-major A operand (M = 128 rows, K = d) and
-// V^T, split into a high and a low bf16 half, as the K-major B operand, into one of two
+// X^T, split into a high and a low bf16 half, as the K-major B operand, into one of two
 // accumulators in tensor memory; warps 0-3 read the finished accumulator (one row per
 // thread), round to bf16 and store the rows, while the next tile is being multiplied
 // into the other accumulator.  H is read from HBM once and never passes through registers.
@@ -20,7 +21,7 @@ namespace {
 
 constexpr int kTileRows = kGramTileRows;
 constexpr int kEpiThreads = 128, kProducerWarp = 4, kMmaWarp = 5, kThreads = 192;
-constexpr int kAccCols = 64;                 // tensor-memory columns per accumulator
+constexpr int kMaxCols = 128;                // q <= 128 output columns
 constexpr int kErrProducer = 0x41, kErrMma = 0x42, kErrEpilogue = 0x43;
 
 template <int D> struct UsCfg {
@@ -28,8 +29,8 @@ template <int D> struct UsCfg {
   static constexpr int BOX_BYTES = kTileRows * 128;          // 16 KB: 128 rows x 64 bf16
   static constexpr int TILE_BYTES = KB * BOX_BYTES;
   static constexpr int STAGES = (D == 64) ? 6 : 4;
-  static constexpr int V_BYTES = 2 * KB * kTokenSlots * 128; // [2 halves][KB][64 rows][128 B]
-  static constexpr size_t SMEM = (size_t)STAGES * TILE_BYTES + V_BYTES + 1024;
+  // ring + X^T as [2 halves][KB][np rows][128 B] + slack to align to 1024
+  static constexpr size_t smem(int np) { return (size_t)STAGES * TILE_BYTES + (size_t)2 * KB * np * 128 + 1024; }
 };
 
 // byte offset of 16-byte chunk c of row `row` in a [rows][128 B] tile with the 128-byte swizzle
@@ -46,6 +47,7 @@ template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 project_us_umma_kernel(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ V,
                        __nv_bfloat16* __restrict__ US, int N, int r, int chunk_rows) {
+  // V is the per-user matrix X [D][r] and US the output [N][r]; r stands for q here.
   using Cfg = UsCfg<D>;
   constexpr int STAGES = Cfg::STAGES;
   extern __shared__ uint8_t smem_raw[];
@@ -65,6 +67,7 @@ project_us_umma_kernel(const __grid_constant__ CUtensorMap tmap, const float* __
   const int ntiles = (row1 - row0 + kTileRows - 1) / kTileRows;
   const int np = (r + 15) & ~15;              // columns the GEMM runs over (multiple of 16)
   const int v_tile = np * 128;                // bytes of one [np rows][128 B] tile of V^T
+  const int acc_cols = np > 64 ? 128 : 64;    // tensor-memory columns per accumulator
 
   if (tid == 0) {
     s_err = 0;
@@ -73,7 +76,7 @@ project_us_umma_kernel(const __grid_constant__ CUtensorMap tmap, const float* __
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&tmap);
   }
-  if (warp == kMmaWarp) ptx::tmem_alloc(&s_tmem, 2 * kAccCols);
+  if (warp == kMmaWarp) ptx::tmem_alloc(&s_tmem, 2 * acc_cols);
   ptx::tc_fence_before_sync();
   __syncthreads();
   ptx::tc_fence_after_sync();
@@ -138,7 +141,7 @@ project_us_umma_kernel(const __grid_constant__ CUtensorMap tmap, const float* __
           for (int kk = 0; kk < D / 16; ++kk) {
             const uint32_t ha = hbase + (kk / 4) * Cfg::BOX_BYTES + (kk % 4) * 32;
             const uint32_t vb = vbase + (h * Cfg::KB + kk / 4) * v_tile + (kk % 4) * 32;
-            ptx::umma_bf16_ss(tmem + a * kAccCols, ptx::umma_smem_desc(ha, 0, 1024),
+            ptx::umma_bf16_ss(tmem + a * acc_cols, ptx::umma_smem_desc(ha, 0, 1024),
                               ptx::umma_smem_desc(vb, 0, 1024), idesc, (h | kk) != 0);
           }
         ptx::umma_commit(&empty_bar[st]);     // the stage is free once these MMAs have read it
@@ -155,41 +158,30 @@ project_us_umma_kernel(const __grid_constant__ CUtensorMap tmap, const float* __
       // the warp leaves together: the tensor-memory loads below are warp-wide
       if (!__all_sync(0xffffffffu, ptx::mbar_wait(&acc_full[a], (t >> 1) & 1, err, kErrEpilogue))) break;
       ptx::tc_fence_after_sync();
-      uint32_t v0[32], v1[32];
-      ptx::tmem_ld_32x32(tmem + lane_base + a * kAccCols, v0);
-      if (np > 32) ptx::tmem_ld_32x32(tmem + lane_base + a * kAccCols + 32, v1);
-      ptx::tmem_ld_wait();
-      ptx::tc_fence_before_sync();
-      ptx::mbar_arrive(&acc_free[a]);          // the accumulator may be overwritten
       const int n = row0 + t * kTileRows + tid;
-      if (n < N) {
-        __nv_bfloat16* o = US + ((size_t)b * N + n) * r;
-        if (vec) {
-          uint4* o4 = reinterpret_cast<uint4*>(o);
-#pragma unroll
-          for (int c = 0; c < 4; ++c)
-            if (8 * c < r)
-              o4[c] = make_uint4(pack2(__uint_as_float(v0[8 * c]), __uint_as_float(v0[8 * c + 1])),
-                                 pack2(__uint_as_float(v0[8 * c + 2]), __uint_as_float(v0[8 * c + 3])),
-                                 pack2(__uint_as_float(v0[8 * c + 4]), __uint_as_float(v0[8 * c + 5])),
-                                 pack2(__uint_as_float(v0[8 * c + 6]), __uint_as_float(v0[8 * c + 7])));
-          if (np > 32) {
+      __nv_bfloat16* o = US + ((size_t)b * N + (n < N ? n : 0)) * r;
+      for (int c0 = 0; c0 < np; c0 += 32) {
+        uint32_t v[32];
+        ptx::tmem_ld_32x32(tmem + lane_base + a * acc_cols + c0, v);
+        ptx::tmem_ld_wait();
+        if (c0 + 32 >= np) {                     // last chunk read: the accumulator may be overwritten
+          ptx::tc_fence_before_sync();
+          ptx::mbar_arrive(&acc_free[a]);
+        }
+        if (n < N) {
+          if (vec) {
+            uint4* o4 = reinterpret_cast<uint4*>(o + c0);
 #pragma unroll
             for (int c = 0; c < 4; ++c)
-              if (32 + 8 * c < r)
-                o4[4 + c] = make_uint4(pack2(__uint_as_float(v1[8 * c]), __uint_as_float(v1[8 * c + 1])),
-                                       pack2(__uint_as_float(v1[8 * c + 2]), __uint_as_float(v1[8 * c + 3])),
-                                       pack2(__uint_as_float(v1[8 * c + 4]), __uint_as_float(v1[8 * c + 5])),
-                                       pack2(__uint_as_float(v1[8 * c + 6]), __uint_as_float(v1[8 * c + 7])));
-          }
-        } else {
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (i < r) o[i] = __float2bfloat16_rn(__uint_as_float(v0[i]));
-          if (np > 32) {
+              if (c0 + 8 * c < r)
+                o4[c] = make_uint4(pack2(__uint_as_float(v[8 * c]), __uint_as_float(v[8 * c + 1])),
+                                   pack2(__uint_as_float(v[8 * c + 2]), __uint_as_float(v[8 * c + 3])),
+                                   pack2(__uint_as_float(v[8 * c + 4]), __uint_as_float(v[8 * c + 5])),
+                                   pack2(__uint_as_float(v[8 * c + 6]), __uint_as_float(v[8 * c + 7])));
+          } else {
 #pragma unroll
             for (int i = 0; i < 32; ++i)
-              if (32 + i < r) o[32 + i] = __float2bfloat16_rn(__uint_as_float(v1[i]));
+              if (c0 + i < r) o[c0 + i] = __float2bfloat16_rn(__uint_as_float(v[i]));
           }
         }
       }
@@ -203,7 +195,7 @@ project_us_umma_kernel(const __grid_constant__ CUtensorMap tmap, const float* __
   }
   ptx::tc_fence_before_sync();
   __syncthreads();
-  if (warp == kMmaWarp) ptx::tmem_dealloc(tmem, 2 * kAccCols);
+  if (warp == kMmaWarp) ptx::tmem_dealloc(tmem, 2 * acc_cols);
 }
 
 template <int D>
@@ -214,11 +206,12 @@ cudaError_t launch_d(int B, int N, int r, const void* H, const float* V, void* U
   if (!encode_tmap_bf16_3d(&tmap, H, D, (uint64_t)N, (uint64_t)B, (uint64_t)D * 2, (uint64_t)N * D * 2, 64,
                            kTileRows))
     return cudaErrorInvalidValue;
+  const size_t smem = Cfg::smem((r + 15) & ~15);
   cudaError_t e = cudaFuncSetAttribute(project_us_umma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)Cfg::SMEM);
+                                       (int)Cfg::smem(kMaxCols));
   if (e != cudaSuccess) return e;
   const dim3 grid(plan.splits, B), block(kThreads);
-  project_us_umma_kernel<D><<<grid, block, Cfg::SMEM, st>>>(tmap, V, static_cast<__nv_bfloat16*>(US), N, r,
+  project_us_umma_kernel<D><<<grid, block, smem, st>>>(tmap, V, static_cast<__nv_bfloat16*>(US), N, r,
                                                            plan.chunk_tiles * kTileRows);
   return cudaGetLastError();
 }
@@ -226,7 +219,7 @@ cudaError_t launch_d(int B, int N, int r, const void* H, const float* V, void* U
 }  // namespace
 
 bool project_us_umma_supported(int N, int d, int r, solar_dtype_t dt) {
-  return dt == SOLAR_BF16 && (d == 64 || d == 128) && N >= kTileRows && r >= 1 && r <= kTokenSlots;
+  return dt == SOLAR_BF16 && (d == 64 || d == 128) && N >= kTileRows && r >= 1 && r <= kMaxCols;
 }
 
 cudaError_t launch_project_us_umma(int B, int N, int d, int r, const void* H, const float* V, void* US,

@@ -186,6 +186,27 @@ solar_status_t solar_svd_attention_fwd(int B, int M, int N, int d, int r, solar_
   return solar_attn_apply(B, M, d, r, dt, C, flags, O, workspace, workspace_bytes, stream);
 }
 
+solar_status_t solar_svd_backward(int B, int N, int d, int r, solar_dtype_t dt, const void* H,
+                                  const float* S, const float* V, const float* dS, const float* dV,
+                                  float eps_rel, void* dH, void* workspace, size_t workspace_bytes,
+                                  void* stream) {
+  SOLAR_TRY(check_dims(B, 0, N, d, r, dt));
+  if (!(eps_rel >= 0.f)) return SOLAR_ERR_INVALID_ARG;
+  if (B == 0) return SOLAR_OK;
+  SOLAR_TRY(check_ptr(H));
+  SOLAR_TRY(check_ptr(S));
+  SOLAR_TRY(check_ptr(V));
+  SOLAR_TRY(check_ptr(dS));
+  SOLAR_TRY(check_ptr(dV));
+  SOLAR_TRY(check_ptr(dH));
+  SOLAR_TRY(check_ws(workspace, workspace_bytes, (size_t)B * d * d * sizeof(float)));
+  const cudaStream_t st = static_cast<cudaStream_t>(stream);
+  float* K = static_cast<float*>(workspace);
+  SOLAR_TRY(from_cuda(launch_svd_grad(B, d, r, S, V, dS, dV, eps_rel, K, st)));
+  // dH_b = H_b K_b: the right-multiplication kernel of the left factor, with q = d columns
+  return from_cuda(launch_project_us(B, N, d, d, dt, H, K, dH, st));
+}
+
 solar_status_t solar_factored_softmax_attention_fwd(int B, int M, int N, int d, int r, solar_dtype_t dt,
                                                     const void* C, const void* US, const float* V,
                                                     const void* Wq, const void* Wk, const void* Wv,

@@ -96,6 +96,8 @@ cudaError_t launch_eig(int B, int d, int r, solar_dtype_t dt, int route, const f
 int eig_subspace_dim(int d, int r);
 cudaError_t launch_project_us(int B, int N, int d, int r, solar_dtype_t dt, const void* H,
                               const float* V, void* US, cudaStream_t st);
+cudaError_t launch_svd_grad(int B, int d, int r, const float* S, const float* V, const float* dS,
+                            const float* dV, float eps_rel, float* K, cudaStream_t st);
 bool project_us_umma_supported(int N, int d, int r, solar_dtype_t dt);
 cudaError_t launch_project_us_umma(int B, int N, int d, int r, const void* H, const float* V, void* US,
                                    cudaStream_t st);

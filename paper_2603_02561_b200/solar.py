@@ -36,6 +36,8 @@ SIGNATURES = {
     "solar_eig_from_partials_ex": (_c_int, [_c_int] * 4 + [_c_int, _c_int] + [_c_vp] * 4 +
                                    [_c_vp, _c_size, _c_vp]),
     "solar_project_us": (_c_int, [_c_int] * 4 + [_c_int] + [_c_vp] * 3 + [_c_vp]),
+    "solar_svd_backward": (_c_int, [_c_int] * 4 + [_c_int] + [_c_vp] * 5 + [_c_float] + [_c_vp] * 2 +
+                           [_c_size, _c_vp]),
     "solar_attn_prepare": (_c_int, [_c_int] * 3 + [_c_int] + [_c_vp] * 5 + [_c_float, _c_vp, _c_size, _c_vp]),
     "solar_factored_softmax_attention_fwd": (_c_int, [_c_int] * 5 + [_c_int] + [_c_vp] * 6 +
                                              [_c_float, _c_vp, _c_vp, _c_size, _c_vp]),
@@ -218,6 +220,15 @@ def project_us(H, V, US, stream=None):
     r = V.shape[2]
     _check(lib().solar_project_us(B, N, d, r, dtype_code(H.dtype), _ptr(H), _ptr(V), _ptr(US),
                                   _stream(stream)), "solar_project_us")
+
+
+def svd_backward(H, S, V, dS, dV, dH, workspace, eps_rel=0.0, stream=None):
+    """dH = U [diag(dS) + 2 Sigma sym(F o (dV^T V))] V^T with U = H V Sigma^-1 (Eq. 13-15)."""
+    B, N, d = H.shape
+    r = V.shape[2]
+    _check(lib().solar_svd_backward(B, N, d, r, dtype_code(H.dtype), _ptr(H), _ptr(S), _ptr(V), _ptr(dS),
+                                    _ptr(dV), float(eps_rel), _ptr(dH), _ptr(workspace), workspace.numel(),
+                                    _stream(stream)), "solar_svd_backward")
 
 
 def attn_prepare(S, V, Wq, Wk, Wv, scale, workspace, stream=None):
