@@ -199,6 +199,32 @@ solar_status_t solar_svd_backward(int B, int N, int d, int r, solar_dtype_t dt, 
                                   void* stream);
 
 /* ------------------------------------------------------------------------- *
+ * Backward pass of solar_svd_attention_fwd: the chain rule through Eq. 11-12 (the
+ * paper prints the SVD's gradient, Eq. 13-15, and leaves this part to calculus).
+ * Given dO = dL/dO it returns the gradients with respect to every input of the
+ * forward call; dS and dV then go to solar_svd_backward for dL/dH.
+ *
+ *   C, S, V, Wq, Wk, Wv, scale, flags: exactly as given to solar_svd_attention_fwd
+ *   dO   [B,M,d] dt  (in)
+ *   dC   [B,M,d] dt  (out)
+ *   dWq, dWk, dWv [d,d] f32 (out)  summed over the B users (overwritten, not accumulated)
+ *   dS   [B,r]   f32 (out)  dL/dSigma        dV [B,d,r] f32 (out)  dL/dV
+ *   workspace: solar_backward_workspace_bytes() of the same sizes; contents undefined on
+ *   return.  The scores and probabilities are recomputed from C, never stored.
+ * Sums over candidates and over users run in a fixed order: the results are
+ * reproducible bit for bit.  N is accepted for a uniform signature and ignored.
+ * ------------------------------------------------------------------------- */
+size_t solar_backward_workspace_bytes(int B, int M, int N, int d, int r, solar_dtype_t dt);
+
+solar_status_t solar_svd_attention_bwd(int B, int M, int N, int d, int r, solar_dtype_t dt,
+                                       const void* C, const float* S, const float* V,
+                                       const void* Wq, const void* Wk, const void* Wv,
+                                       float scale, unsigned flags, const void* dO,
+                                       void* dC, float* dWq, float* dWk, float* dWv,
+                                       float* dS, float* dV,
+                                       void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------- *
  * Softmax attention over the N history positions, evaluated through the factors:
  *   O = softmax_rows( scale * (C W_Q W_K^T V) (U Sigma)^T ) (U Sigma) (V^T W_V)    [M,d]
  * With H = U Sigma V^T of rank <= r this equals the softmax attention of Eq. 6-7,

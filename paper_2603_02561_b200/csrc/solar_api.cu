@@ -186,6 +186,45 @@ solar_status_t solar_svd_attention_fwd(int B, int M, int N, int d, int r, solar_
   return solar_attn_apply(B, M, d, r, dt, C, flags, O, workspace, workspace_bytes, stream);
 }
 
+size_t solar_backward_workspace_bytes(int B, int M, int N, int d, int r, solar_dtype_t dt) {
+  if (check_dims(B, M, N, d, r, dt) != SOLAR_OK) return 0;
+  const size_t a = bwd_ws_layout(B, M, d, r).total, k = (size_t)B * d * d * sizeof(float);
+  return a > k ? a : k;
+}
+
+solar_status_t solar_svd_attention_bwd(int B, int M, int N, int d, int r, solar_dtype_t dt,
+                                       const void* C, const float* S, const float* V,
+                                       const void* Wq, const void* Wk, const void* Wv,
+                                       float scale, unsigned flags, const void* dO,
+                                       void* dC, float* dWq, float* dWk, float* dWv,
+                                       float* dS, float* dV,
+                                       void* workspace, size_t workspace_bytes, void* stream) {
+  (void)N;
+  SOLAR_TRY(check_dims(B, M, r, d, r, dt));
+  if (flags & ~(unsigned)SOLAR_FLAG_NO_SOFTMAX) return SOLAR_ERR_INVALID_ARG;
+  if (B == 0) return SOLAR_OK;
+  if (M > 0) { SOLAR_TRY(check_ptr(C)); SOLAR_TRY(check_ptr(dO)); SOLAR_TRY(check_ptr(dC)); }
+  SOLAR_TRY(check_ptr(S));
+  SOLAR_TRY(check_ptr(V));
+  SOLAR_TRY(check_ptr(Wq));
+  SOLAR_TRY(check_ptr(Wk));
+  SOLAR_TRY(check_ptr(Wv));
+  SOLAR_TRY(check_ptr(dWq));
+  SOLAR_TRY(check_ptr(dWk));
+  SOLAR_TRY(check_ptr(dWv));
+  SOLAR_TRY(check_ptr(dS));
+  SOLAR_TRY(check_ptr(dV));
+  const BwdWs bl = bwd_ws_layout(B, M, d, r);
+  SOLAR_TRY(check_ws(workspace, workspace_bytes, bl.total));
+  const cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const AttnWs lay = attn_ws_layout(d, r);
+  char* ws = static_cast<char*>(workspace);
+  // T_b and Value_r as in the forward call
+  SOLAR_TRY(from_cuda(launch_attn_prepare(B, d, r, dt, S, V, Wq, Wk, Wv, scale, ws, lay, st)));
+  return from_cuda(launch_attn_bwd(B, M, d, r, dt, C, dO, S, V, Wq, Wk, Wv, scale, flags, dC, dWq, dWk, dWv,
+                                   dS, dV, ws, lay, bl, st));
+}
+
 solar_status_t solar_svd_backward(int B, int N, int d, int r, solar_dtype_t dt, const void* H,
                                   const float* S, const float* V, const float* dS, const float* dV,
                                   float eps_rel, void* dH, void* workspace, size_t workspace_bytes,

@@ -84,6 +84,40 @@ inline size_t attn_ws_bytes(int B, int d, int r) {
   return attn_ws_layout(d, r).per_user * (size_t)B;
 }
 
+// Backward pass of the attention: how the M candidates of a user are cut into row chunks
+// (one CTA each; every chunk leaves one partial of the two per-user reductions over M),
+// and the workspace behind the attention call's own segments:
+//   part [B][chunks][2][d][64] fp32   partial dT (= C^T dS) and dValue_r^T (= dO^T P)
+//   dw   [B][3][d][d]          fp32   per-user contributions to dW_Q, dW_K, dW_V
+struct BwdPlan {
+  int rows_per_cta;   // a multiple of 32
+  int chunks;
+};
+inline BwdPlan bwd_plan(int B, int M) {
+  BwdPlan p;
+  const int b = B > 0 ? B : 1;
+  int want = (2 * kNumSMs + b - 1) / b;               // about two CTAs per SM over all users
+  const int max_chunks = (M + 31) / 32 > 0 ? (M + 31) / 32 : 1;
+  if (want > max_chunks) want = max_chunks;
+  if (want < 1) want = 1;
+  p.rows_per_cta = (((M + want - 1) / want + 31) / 32) * 32;
+  if (p.rows_per_cta < 32) p.rows_per_cta = 32;
+  p.chunks = (M + p.rows_per_cta - 1) / p.rows_per_cta;
+  if (p.chunks < 1) p.chunks = 1;
+  return p;
+}
+struct BwdWs {
+  size_t part_off, dw_off, total;
+};
+inline BwdWs bwd_ws_layout(int B, int M, int d, int r) {
+  BwdWs w;
+  const BwdPlan p = bwd_plan(B, M);
+  w.part_off = align_up(attn_ws_bytes(B, d, r), 256);
+  w.dw_off = w.part_off + align_up((size_t)B * p.chunks * 2 * d * kTokenSlots * sizeof(float), 256);
+  w.total = w.dw_off + align_up((size_t)B * 3 * d * d * sizeof(float), 256);
+  return w;
+}
+
 // ---- launchers (one per kernel file) --------------------------------------
 cudaError_t launch_gram_simt(int B, int N, int d, solar_dtype_t dt, const void* H, float* gpart,
                              int* status, const GramPlan& plan, cudaStream_t st);
@@ -98,6 +132,11 @@ cudaError_t launch_project_us(int B, int N, int d, int r, solar_dtype_t dt, cons
                               const float* V, void* US, cudaStream_t st);
 cudaError_t launch_svd_grad(int B, int d, int r, const float* S, const float* V, const float* dS,
                             const float* dV, float eps_rel, float* K, cudaStream_t st);
+cudaError_t launch_attn_bwd(int B, int M, int d, int r, solar_dtype_t dt, const void* C, const void* dO,
+                            const float* S, const float* V, const void* Wq, const void* Wk, const void* Wv,
+                            float scale, unsigned flags, void* dC, float* dWq, float* dWk, float* dWv,
+                            float* dS, float* dV, char* ws, const AttnWs& lay, const BwdWs& bl,
+                            cudaStream_t st);
 bool project_us_umma_supported(int N, int d, int r, solar_dtype_t dt);
 cudaError_t launch_project_us_umma(int B, int N, int d, int r, const void* H, const float* V, void* US,
                                    cudaStream_t st);

@@ -38,6 +38,9 @@ SIGNATURES = {
     "solar_project_us": (_c_int, [_c_int] * 4 + [_c_int] + [_c_vp] * 3 + [_c_vp]),
     "solar_svd_backward": (_c_int, [_c_int] * 4 + [_c_int] + [_c_vp] * 5 + [_c_float] + [_c_vp] * 2 +
                            [_c_size, _c_vp]),
+    "solar_backward_workspace_bytes": (_c_size, [_c_int] * 5 + [_c_int]),
+    "solar_svd_attention_bwd": (_c_int, [_c_int] * 5 + [_c_int] + [_c_vp] * 6 + [_c_float, _c_uint] +
+                                [_c_vp] * 7 + [_c_vp, _c_size, _c_vp]),
     "solar_attn_prepare": (_c_int, [_c_int] * 3 + [_c_int] + [_c_vp] * 5 + [_c_float, _c_vp, _c_size, _c_vp]),
     "solar_factored_softmax_attention_fwd": (_c_int, [_c_int] * 5 + [_c_int] + [_c_vp] * 6 +
                                              [_c_float, _c_vp, _c_vp, _c_size, _c_vp]),
@@ -220,6 +223,33 @@ def project_us(H, V, US, stream=None):
     r = V.shape[2]
     _check(lib().solar_project_us(B, N, d, r, dtype_code(H.dtype), _ptr(H), _ptr(V), _ptr(US),
                                   _stream(stream)), "solar_project_us")
+
+
+def backward_workspace_bytes(B, M, N, d, r, dtype) -> int:
+    return int(lib().solar_backward_workspace_bytes(B, M, N, d, r, dtype_code(dtype)))
+
+
+def alloc_backward_workspace(B, M, N, d, r, dtype, device="cuda") -> torch.Tensor:
+    return torch.empty(max(backward_workspace_bytes(B, M, N, d, r, dtype), 256), dtype=torch.uint8, device=device)
+
+
+def svd_attention_bwd(C, S, V, Wq, Wk, Wv, scale, dO, workspace, flags=0, stream=None):
+    """solar_svd_attention_bwd: gradients of the forward call's inputs given dO.
+    Returns dC[B,M,d], dWq, dWk, dWv [d,d] f32, dS[B,r], dV[B,d,r]."""
+    B, M, d = C.shape
+    r = S.shape[1]
+    _need(dO, (B, M, d), C.dtype, "dO")
+    dev = C.device
+    dC = torch.empty_like(C)
+    dWq, dWk, dWv = (torch.empty(d, d, dtype=torch.float32, device=dev) for _ in range(3))
+    dS = torch.empty(B, r, dtype=torch.float32, device=dev)
+    dV = torch.empty(B, d, r, dtype=torch.float32, device=dev)
+    _check(lib().solar_svd_attention_bwd(B, M, max(r, 1), d, r, dtype_code(C.dtype), _ptr(C), _ptr(S), _ptr(V),
+                                         _ptr(Wq), _ptr(Wk), _ptr(Wv), float(scale), int(flags), _ptr(dO),
+                                         _ptr(dC), _ptr(dWq), _ptr(dWk), _ptr(dWv), _ptr(dS), _ptr(dV),
+                                         _ptr(workspace), workspace.numel(), _stream(stream)),
+           "solar_svd_attention_bwd")
+    return dC, dWq, dWk, dWv, dS, dV
 
 
 def svd_backward(H, S, V, dS, dV, dH, workspace, eps_rel=0.0, stream=None):

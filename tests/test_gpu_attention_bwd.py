@@ -1,0 +1,109 @@
+"""solar_svd_attention_bwd (chain rule through Eq. 11-12) against the CPU oracle on the
+factors the CUDA factorization returns, element by element; the whole backward pass
+(attention part, then Eq. 13-15) against the oracle's; reproducibility bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as o
+from oracle import svd_attention_backward as ob
+from paper_2603_02561_b200 import solar
+from paper_2603_02561_b200 import workloads as wl
+
+import parity_harness as ph
+
+pytestmark = pytest.mark.gpu
+
+CASES = [
+    # workload, flags
+    (wl.CONFIGS["c1"], 0),                                           # fp32 storage, d = 32
+    (wl.CONFIGS["c1"], solar.FLAG_NO_SOFTMAX),
+    (wl.CONFIGS["c2"].with_(B=4, M=300), 0),                         # several chunks, ragged last batch
+    (wl.CONFIGS["c2"].with_(B=3, M=5), 0),                           # fewer rows than one batch
+    (wl.CONFIGS["c3"].with_(B=2, N=2048, M=700), 0),
+    (wl.CONFIGS["c3"].with_(B=2, N=2048, M=257, r=27), solar.FLAG_NO_SOFTMAX),
+    (wl.CONFIGS["c4"].with_(B=2, N=512, M=200), 0),                  # d = 128, r = 64
+]
+
+
+def _f64(t):
+    return t.float().cpu().numpy().astype(np.float64)
+
+
+def _setup(w, seed):
+    inp = wl.generate(w)
+    tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    H = ph.to_device(inp["H"], w.dtype); C = ph.to_device(inp["C"], w.dtype)
+    Wq, Wk, Wv = (ph.to_device(inp[k], w.dtype) for k in ("Wq", "Wk", "Wv"))
+    B, N, d = H.shape
+    ws = solar.alloc_workspace(B, w.M, N, d, w.r, tdt)
+    S, V = solar.lowrank_factor(H, w.r, workspace=ws)
+    g = torch.Generator().manual_seed(seed)
+    dO = torch.randn(B, w.M, d, generator=g).to(tdt).cuda()
+    bws = solar.alloc_backward_workspace(B, w.M, N, d, w.r, tdt)
+    return inp, H, C, Wq, Wk, Wv, S, V, dO, bws
+
+
+def _rel(got, ref):
+    return np.abs(got - ref).max() / max(np.abs(ref).max(), 1e-300)
+
+
+@pytest.mark.parametrize("w,flags", CASES, ids=[f"{c[0].name}_M{c[0].M}_r{c[0].r}_f{c[1]}" for c in CASES])
+def test_attention_bwd_matches_oracle(w, flags):
+    inp, H, C, Wq, Wk, Wv, S, V, dO, bws = _setup(w, seed=w.M + w.r)
+    bws.fill_(0xFF)
+    dC, dWq, dWk, dWv, dS, dV = solar.svd_attention_bwd(C, S, V, Wq, Wk, Wv, inp["scale"], dO, bws, flags=flags)
+    torch.cuda.synchronize()
+    S64, V64, dO64 = _f64(S), _f64(V), _f64(dO)
+    B = S64.shape[0]
+    sums = {k: 0.0 for k in ("dWq", "dWk", "dWv")}
+    out_tol = 1e-2 if w.dtype == "bf16" else 1e-4       # dC is rounded to the storage type
+    for k in range(B):
+        g = ob.svd_attention_backward(inp["C"][k].astype(np.float64), S64[k], V64[k],
+                                      *(inp[n].astype(np.float64) for n in ("Wq", "Wk", "Wv")),
+                                      inp["scale"], dO64[k], softmax=not flags)
+        assert o.max_rel_err_rows(_f64(dC[k]), g["dC"]) <= out_tol
+        assert _rel(_f64(dS[k]), g["ds"]) <= 1e-4
+        assert _rel(_f64(dV[k]), g["dV"]) <= 1e-4
+        for n in sums:
+            sums[n] = sums[n] + g[n]
+    for n, t in (("dWq", dWq), ("dWk", dWk), ("dWv", dWv)):
+        assert _rel(_f64(t), sums[n]) <= 1e-4, n
+
+
+def test_whole_backward_pass_matches_oracle():
+    w = wl.CONFIGS["c3"].with_(B=2, N=1500, M=400)
+    inp, H, C, Wq, Wk, Wv, S, V, dO, bws = _setup(w, seed=11)
+    dC, dWq, dWk, dWv, dS, dV = solar.svd_attention_bwd(C, S, V, Wq, Wk, Wv, inp["scale"], dO, bws)
+    dH = torch.empty_like(H)
+    solar.svd_backward(H, S, V, dS, dV, dH, bws)
+    torch.cuda.synchronize()
+    S64, V64, dO64 = _f64(S), _f64(V), _f64(dO)
+    for k in range(2):
+        g = ob.svd_attention_backward_full(inp["H"][k].astype(np.float64), inp["C"][k].astype(np.float64),
+                                           S64[k], V64[k], *(inp[n].astype(np.float64) for n in ("Wq", "Wk", "Wv")),
+                                           inp["scale"], dO64[k])
+        assert _rel(_f64(dH[k]), g["dH"]) <= 2.0 ** -7
+
+
+def test_attention_bwd_is_reproducible_bit_for_bit():
+    w = wl.CONFIGS["c2"].with_(B=4, M=1000)
+    inp, H, C, Wq, Wk, Wv, S, V, dO, bws = _setup(w, seed=3)
+    a = solar.svd_attention_bwd(C, S, V, Wq, Wk, Wv, inp["scale"], dO, bws)
+    torch.cuda.synchronize()
+    bws2 = torch.zeros_like(bws)
+    b = solar.svd_attention_bwd(C, S, V, Wq, Wk, Wv, inp["scale"], dO, bws2)
+    torch.cuda.synchronize()
+    for x, y in zip(a, b):
+        assert torch.equal(x.view(torch.uint8), y.view(torch.uint8))
+
+
+def test_attention_bwd_argument_checks():
+    w = wl.CONFIGS["c1"]
+    inp, H, C, Wq, Wk, Wv, S, V, dO, bws = _setup(w, seed=1)
+    with pytest.raises(solar.SolarError) as e:
+        solar.svd_attention_bwd(C, S, V, Wq, Wk, Wv, inp["scale"], dO, bws[:128])
+    assert e.value.status == solar.ERR_WORKSPACE
+    with pytest.raises(solar.SolarError) as e:
+        solar.svd_attention_bwd(C, S, V, Wq, Wk, Wv, inp["scale"], dO, bws, flags=2)
+    assert e.value.status == solar.ERR_INVALID_ARG
