@@ -6,10 +6,11 @@
 //   dW_Q = scale dT Key_r,   dKey_r = scale dT^T W_Q,
 //   dA = dKey_r W_K^T + dValue_r W_V^T,   A = Sigma V^T,
 //   dW_K = A^T dKey_r,   dW_V = A^T dValue_r,   dSigma_i = sum_k dA_ik V_ki,   dV_ki = dA_ik sigma_i.
-// Three kernels: the streaming one (one CTA per chunk of candidate rows; recomputes S and P,
-// writes dC and a partial of dT and dValue_r^T), a per-user one (sums the partials in chunk
-// order, runs the small chain, writes dSigma, dV and this user's dW contributions) and a
-// sum over users in user order.  FFMA arithmetic in fp32 for every shape and storage type.
+// Four kernels: the streaming one (one CTA per chunk of candidate rows; recomputes S and P,
+// writes dC and a partial of dT and dValue_r^T), the sum of the partials in chunk order, a
+// per-user one (the small chain; writes dSigma, dV and this user's dW contributions) and a
+// sum over users in user order.  The streaming kernel here is the FFMA one (fp32 storage,
+// d = 32); bf16 storage with d = 64 or 128 takes the tensor-core kernel instead.
 #include <math.h>
 
 #include "solar_internal.cuh"
@@ -154,6 +155,8 @@ attn_bwd_rows_kernel(const T* __restrict__ C, const T* __restrict__ dO, T* __res
 }
 
 // Per-user chain from dT and dValue_r to dSigma, dV and this user's dW contributions.
+// Each weight matrix is staged in shared memory (fp32, odd pitch) when it is needed: W_K for
+// Key_r, W_Q for dKey_r, then W_K and W_V again for dA, where they are read along their rows.
 template <typename T, int D>
 __global__ void __launch_bounds__(kThreads)
 attn_bwd_user_kernel(const float* __restrict__ part, int chunks, const float* __restrict__ S,
@@ -161,33 +164,45 @@ attn_bwd_user_kernel(const float* __restrict__ part, int chunks, const float* __
                      const T* __restrict__ Wv, float scale, int r, float* __restrict__ dS,
                      float* __restrict__ dV, float* __restrict__ dw) {
   extern __shared__ __align__(16) float sm[];
-  float* dT = sm;                       // [D][kRP]   dT[k][i]
-  float* dVT = dT + D * kRP;            // [D][kRP]   dValue_r^T[j][i]
-  float* A = dVT + D * kRP;             // [kRP][D]   Sigma V^T
+  constexpr int LR = kRP + 1;           // odd pitch: dT and dValue_r^T are read along both indices
+  constexpr int LW = D + 1;             // odd pitch of the staged weight matrix
+  float* dT = sm;                       // [D][LR]    dT[k][i]
+  float* dVT = dT + D * LR;             // [D][LR]    dValue_r^T[j][i]
+  float* A = dVT + D * LR;              // [kRP][D]   Sigma V^T, at the end dA
   float* X = A + kRP * D;               // [kRP][D]   Key_r, then dKey_r
-  float* dA = X + kRP * D;              // [kRP][D]
+  float* Ws = X + kRP * D;              // [D][LW]    the weight matrix in use
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-  // partials in chunk order
-  for (int e = tid; e < 2 * D * kRP; e += kThreads) {
-    float acc = 0.f;
-    for (int c = 0; c < chunks; ++c) acc += part[((size_t)b * chunks + c) * 2 * D * kRP + e];
-    dT[e] = acc;                        // dVT follows dT in shared memory
-  }
+  auto stage = [&](const T* __restrict__ W) {
+    constexpr int VE = Vec16<T>::kElems;
+    for (int v = tid; v < D * D / VE; v += kThreads) {
+      float tmp[VE];
+      Vec16<T>::load(W + (size_t)v * VE, tmp);
+      const int k = (v * VE) / D, j = (v * VE) % D;
+#pragma unroll
+      for (int e = 0; e < VE; ++e) Ws[k * LW + j + e] = tmp[e];
+    }
+  };
+
+  stage(Wk);
+  // the partials, summed into the first chunk's slot by sum_chunks_kernel
+  for (int e = tid; e < 2 * D * kRP; e += kThreads)
+    dT[(e / kRP) * LR + e % kRP] = part[(size_t)b * chunks * 2 * D * kRP + e];   // dVT follows dT in shared memory
   for (int e = tid; e < kRP * D; e += kThreads) {
-    const int i = e / D, k = e % D;
-    A[e] = i < r ? S[(size_t)b * r + i] * V[((size_t)b * D + k) * r + i] : 0.f;
+    const int k = e / kRP, i = e % kRP;   // V is read along its rows
+    A[i * D + k] = i < r ? S[(size_t)b * r + i] * V[((size_t)b * D + k) * r + i] : 0.f;
   }
   __syncthreads();
   // Key_r[i][j] = sum_k A[i][k] W_K[k][j]; lanes run over j
   for (int e = tid; e < r * D; e += kThreads) {
     const int i = e / D, j = e % D;
     float acc = 0.f;
-#pragma unroll 4
-    for (int k = 0; k < D; ++k) acc = fmaf(A[i * D + k], to_f32<T>(Wk[k * D + j]), acc);
+#pragma unroll 8
+    for (int k = 0; k < D; ++k) acc = fmaf(A[i * D + k], Ws[k * LW + j], acc);
     X[e] = acc;
   }
   __syncthreads();
+  stage(Wq);
   float* dWq = dw + (size_t)b * 3 * D * D;
   float* dWk = dWq + D * D;
   float* dWv = dWk + D * D;
@@ -195,7 +210,8 @@ attn_bwd_user_kernel(const float* __restrict__ part, int chunks, const float* __
   for (int e = tid; e < D * D; e += kThreads) {
     const int k = e / D, j = e % D;
     float acc = 0.f;
-    for (int i = 0; i < r; ++i) acc = fmaf(dT[k * kRP + i], X[i * D + j], acc);
+#pragma unroll 4
+    for (int i = 0; i < r; ++i) acc = fmaf(dT[k * LR + i], X[i * D + j], acc);
     dWq[e] = scale * acc;
   }
   __syncthreads();
@@ -203,35 +219,56 @@ attn_bwd_user_kernel(const float* __restrict__ part, int chunks, const float* __
   for (int e = tid; e < r * D; e += kThreads) {
     const int i = e / D, j = e % D;
     float acc = 0.f;
-#pragma unroll 4
-    for (int k = 0; k < D; ++k) acc = fmaf(dT[k * kRP + i], to_f32<T>(Wq[k * D + j]), acc);
+#pragma unroll 8
+    for (int k = 0; k < D; ++k) acc = fmaf(dT[k * LR + i], Ws[k * LW + j], acc);
     X[e] = scale * acc;
   }
   __syncthreads();
+  stage(Wk);
   // dW_K[k][j] = sum_i A[i][k] dKey_r[i][j],  dW_V[k][j] = sum_i A[i][k] dValue_r[i][j]
   for (int e = tid; e < D * D; e += kThreads) {
     const int k = e / D, j = e % D;
     float ak = 0.f, av = 0.f;
+#pragma unroll 4
     for (int i = 0; i < r; ++i) {
       const float a = A[i * D + k];
       ak = fmaf(a, X[i * D + j], ak);
-      av = fmaf(a, dVT[j * kRP + i], av);
+      av = fmaf(a, dVT[j * LR + i], av);
     }
     dWk[e] = ak;
     dWv[e] = av;
   }
-  // dA[i][k] = sum_j dKey_r[i][j] W_K[k][j] + dValue_r[i][j] W_V[k][j]: one warp per entry,
-  // lanes run over j (rows of the weights are read as they are stored)
-  for (int e = warp; e < r * D; e += kWarps) {
-    const int i = e / D, k = e % D;
-    float acc = 0.f;
-    for (int j = lane; j < D; j += 32)
-      acc = fmaf(X[i * D + j], to_f32<T>(Wk[k * D + j]), fmaf(dVT[j * kRP + i], to_f32<T>(Wv[k * D + j]), acc));
+  __syncthreads();
+  // dA[i][k] = sum_j dKey_r[i][j] W_K[k][j] + dValue_r[i][j] W_V[k][j]; lanes run over k.
+  // Each thread keeps its entries in registers across the two staged matrices; dA then
+  // takes the place of A.
+  constexpr int QA = kRP * D / kThreads;
+  float acc_a[QA];
 #pragma unroll
-    for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) dA[e] = acc;
+  for (int q = 0; q < QA; ++q) {
+    const int e = tid + q * kThreads, i = e / D, k = e % D;
+    float acc = 0.f;
+    if (i < r) {
+#pragma unroll 8
+      for (int j = 0; j < D; ++j) acc = fmaf(X[i * D + j], Ws[k * LW + j], acc);
+    }
+    acc_a[q] = acc;
   }
   __syncthreads();
+  stage(Wv);
+  __syncthreads();
+#pragma unroll
+  for (int q = 0; q < QA; ++q) {
+    const int e = tid + q * kThreads, i = e / D, k = e % D;
+    float acc = acc_a[q];
+    if (i < r) {
+#pragma unroll 8
+      for (int j = 0; j < D; ++j) acc = fmaf(dVT[j * LR + i], Ws[k * LW + j], acc);
+    }
+    A[e] = acc;
+  }
+  __syncthreads();
+  const float* dA = A;
   // dSigma_i = sum_k dA[i][k] V[k][i],  dV[k][i] = dA[i][k] sigma_i
   for (int i = warp; i < r; i += kWarps) {
     float acc = 0.f;
@@ -244,6 +281,16 @@ attn_bwd_user_kernel(const float* __restrict__ part, int chunks, const float* __
     const int k = e / r, i = e % r;
     dV[(size_t)b * D * r + e] = dA[i * D + k] * S[(size_t)b * r + i];
   }
+}
+
+// part[b][0][e] = sum over the chunks (in chunk order) of part[b][c][e]
+__global__ void sum_chunks_kernel(float* __restrict__ part, int chunks, int n) {
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= n) return;
+  float* p = part + (size_t)blockIdx.y * chunks * n + e;
+  float acc = 0.f;
+  for (int c = 0; c < chunks; ++c) acc += p[(size_t)c * n];
+  p[0] = acc;
 }
 
 // out[w][e] = sum over users (in user order) of dw[b][w][e]
@@ -262,22 +309,39 @@ cudaError_t launch_td(int B, int M, int r, const void* C, const void* dO, const 
                       const void* Wq, const void* Wk, const void* Wv, float scale, unsigned flags, void* dC,
                       float* dWq, float* dWk, float* dWv, float* dS, float* dV, char* ws, const AttnWs& lay,
                       const BwdWs& bl, cudaStream_t st) {
-  const BwdPlan plan = bwd_plan(B, M);
   float* part = reinterpret_cast<float*>(ws + bl.part_off);
   float* dw = reinterpret_cast<float*>(ws + bl.dw_off);
-  const size_t smem_rows = (size_t)(D * (kRP + 1) + D * kRP + 2 * kBatch * D + 2 * kBatch * kRP) * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(attn_bwd_rows_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)smem_rows);
-  if (e != cudaSuccess) return e;
-  attn_bwd_rows_kernel<T, D><<<dim3(plan.chunks, B), kThreads, smem_rows, st>>>(
-      static_cast<const T*>(C), static_cast<const T*>(dO), static_cast<T*>(dC), ws, lay, part, M, r,
-      plan.rows_per_cta, flags);
-  e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
-  const size_t smem_user = (size_t)(2 * D * kRP + 3 * kRP * D) * sizeof(float);
+  int chunks;
+  cudaError_t e;
+  if (attn_bwd_umma_supported(M, D, sizeof(T) == 2 ? SOLAR_BF16 : SOLAR_F32)) {
+    const BwdTilePlan tp = bwd_tile_plan(B, M);
+    chunks = tp.chunks;
+    e = launch_attn_bwd_umma(B, M, D, r, C, dO, flags, dC, part, ws + bl.pk_off, tp.tiles_per_cta, tp.chunks, ws,
+                             lay, st);
+    if (e != cudaSuccess) return e;
+  } else {
+    const BwdPlan plan = bwd_plan(B, M);
+    chunks = plan.chunks;
+    const size_t smem_rows =
+        (size_t)(D * (kRP + 1) + D * kRP + 2 * kBatch * D + 2 * kBatch * kRP) * sizeof(float);
+    e = cudaFuncSetAttribute(attn_bwd_rows_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)smem_rows);
+    if (e != cudaSuccess) return e;
+    attn_bwd_rows_kernel<T, D><<<dim3(plan.chunks, B), kThreads, smem_rows, st>>>(
+        static_cast<const T*>(C), static_cast<const T*>(dO), static_cast<T*>(dC), ws, lay, part, M, r,
+        plan.rows_per_cta, flags);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  if (chunks > 1) {
+    sum_chunks_kernel<<<dim3((2 * D * kRP + 255) / 256, B), 256, 0, st>>>(part, chunks, 2 * D * kRP);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  const size_t smem_user = (size_t)(2 * D * (kRP + 1) + 2 * kRP * D + D * (D + 1)) * sizeof(float);
   e = cudaFuncSetAttribute(attn_bwd_user_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_user);
   if (e != cudaSuccess) return e;
-  attn_bwd_user_kernel<T, D><<<B, kThreads, smem_user, st>>>(part, plan.chunks, S, V, static_cast<const T*>(Wq),
+  attn_bwd_user_kernel<T, D><<<B, kThreads, smem_user, st>>>(part, chunks, S, V, static_cast<const T*>(Wq),
                                                             static_cast<const T*>(Wk), static_cast<const T*>(Wv),
                                                             scale, r, dS, dV, dw);
   e = cudaGetLastError();

@@ -106,15 +106,32 @@ inline BwdPlan bwd_plan(int B, int M) {
   if (p.chunks < 1) p.chunks = 1;
   return p;
 }
+// The tensor-core kernel works on whole 128-row tiles: tiles per CTA and the number of chunks.
+struct BwdTilePlan {
+  int tiles_per_cta, chunks;
+};
+inline BwdTilePlan bwd_tile_plan(int B, int M) {
+  BwdTilePlan p;
+  const int b = B > 0 ? B : 1;
+  const int tiles = (M + 127) / 128 > 0 ? (M + 127) / 128 : 1;
+  int want = (2 * kNumSMs + b - 1) / b;
+  if (want > tiles) want = tiles;
+  p.tiles_per_cta = (tiles + want - 1) / want;
+  p.chunks = (tiles + p.tiles_per_cta - 1) / p.tiles_per_cta;
+  return p;
+}
+//   pk   [B][4][64][d]         bf16   T and Value_r as the tensor-core kernel's extra operands
 struct BwdWs {
-  size_t part_off, dw_off, total;
+  size_t part_off, dw_off, pk_off, total;
 };
 inline BwdWs bwd_ws_layout(int B, int M, int d, int r) {
   BwdWs w;
-  const BwdPlan p = bwd_plan(B, M);
+  const int c1 = bwd_plan(B, M).chunks, c2 = bwd_tile_plan(B, M).chunks;
+  const int chunks = c1 > c2 ? c1 : c2;
   w.part_off = align_up(attn_ws_bytes(B, d, r), 256);
-  w.dw_off = w.part_off + align_up((size_t)B * p.chunks * 2 * d * kTokenSlots * sizeof(float), 256);
-  w.total = w.dw_off + align_up((size_t)B * 3 * d * d * sizeof(float), 256);
+  w.dw_off = w.part_off + align_up((size_t)B * chunks * 2 * d * kTokenSlots * sizeof(float), 256);
+  w.pk_off = w.dw_off + align_up((size_t)B * 3 * d * d * sizeof(float), 256);
+  w.total = w.pk_off + align_up((size_t)B * 4 * kTokenSlots * d * sizeof(__nv_bfloat16), 256);
   return w;
 }
 
@@ -137,6 +154,10 @@ cudaError_t launch_attn_bwd(int B, int M, int d, int r, solar_dtype_t dt, const 
                             float scale, unsigned flags, void* dC, float* dWq, float* dWk, float* dWv,
                             float* dS, float* dV, char* ws, const AttnWs& lay, const BwdWs& bl,
                             cudaStream_t st);
+bool attn_bwd_umma_supported(int M, int d, solar_dtype_t dt);
+cudaError_t launch_attn_bwd_umma(int B, int M, int d, int r, const void* C, const void* dO, unsigned flags,
+                                 void* dC, float* part, void* pk, int tiles_per_cta, int chunks, const char* ws,
+                                 const AttnWs& lay, cudaStream_t st);
 bool project_us_umma_supported(int N, int d, int r, solar_dtype_t dt);
 cudaError_t launch_project_us_umma(int B, int N, int d, int r, const void* H, const float* V, void* US,
                                    cudaStream_t st);

@@ -29,10 +29,10 @@ __global__ void __launch_bounds__(kGradThreads)
 svd_grad_kernel(const float* __restrict__ S, const float* __restrict__ V, const float* __restrict__ dS,
                 const float* __restrict__ dV, float eps_rel, int r, float* __restrict__ K) {
   extern __shared__ __align__(16) float sm[];
-  const int lw = r + 1;                 // pitch of the r x r matrices
-  float* Vs = sm;                       // [D][r]
-  float* dVs = Vs + D * r;              // [D][r]   Vbar
-  float* Pt = dVs + D * r;              // [r][lw]  Vbar^T V
+  const int lw = r | 1;                 // odd pitch: every matrix here is read along rows and along columns
+  float* Vs = sm;                       // [D][lw]
+  float* dVs = Vs + D * lw;             // [D][lw]  Vbar
+  float* Pt = dVs + D * lw;             // [r][lw]  Vbar^T V
   float* W = Pt + r * lw;               // [r][lw]
   float* T1 = W + r * lw;               // [D][lw]  V W
   float* ss = T1 + D * lw;              // [r] sigma
@@ -40,8 +40,9 @@ svd_grad_kernel(const float* __restrict__ S, const float* __restrict__ V, const 
   const int b = blockIdx.x, tid = threadIdx.x;
 
   for (int e = tid; e < D * r; e += kGradThreads) {
-    Vs[e] = V[(size_t)b * D * r + e];
-    dVs[e] = dV[(size_t)b * D * r + e];
+    const int k = e / r, i = e % r;
+    Vs[k * lw + i] = V[(size_t)b * D * r + e];
+    dVs[k * lw + i] = dV[(size_t)b * D * r + e];
   }
   for (int e = tid; e < r; e += kGradThreads) { ss[e] = S[(size_t)b * r + e]; ds[e] = dS[(size_t)b * r + e]; }
   __syncthreads();
@@ -51,7 +52,7 @@ svd_grad_kernel(const float* __restrict__ S, const float* __restrict__ V, const 
     const int i = e / r, j = e % r;
     float acc = 0.f;
 #pragma unroll 4
-    for (int k = 0; k < D; ++k) acc = fmaf(dVs[k * r + i], Vs[k * r + j], acc);
+    for (int k = 0; k < D; ++k) acc = fmaf(dVs[k * lw + i], Vs[k * lw + j], acc);
     Pt[i * lw + j] = acc;
   }
   float smax = 0.f;
@@ -83,7 +84,7 @@ svd_grad_kernel(const float* __restrict__ S, const float* __restrict__ V, const 
     const int k = e / r, j = e % r;
     float acc = 0.f;
 #pragma unroll 4
-    for (int i = 0; i < r; ++i) acc = fmaf(Vs[k * r + i], W[i * lw + j], acc);
+    for (int i = 0; i < r; ++i) acc = fmaf(Vs[k * lw + i], W[i * lw + j], acc);
     T1[k * lw + j] = acc;
   }
   __syncthreads();
@@ -94,7 +95,7 @@ svd_grad_kernel(const float* __restrict__ S, const float* __restrict__ V, const 
     const int k = e / D, l = e % D;
     float acc = 0.f;
 #pragma unroll 4
-    for (int j = 0; j < r; ++j) acc = fmaf(T1[k * lw + j], Vs[l * r + j], acc);
+    for (int j = 0; j < r; ++j) acc = fmaf(T1[k * lw + j], Vs[l * lw + j], acc);
     Kb[e] = acc;
   }
 }
@@ -102,7 +103,7 @@ svd_grad_kernel(const float* __restrict__ S, const float* __restrict__ V, const 
 template <int D>
 cudaError_t launch_d(int B, int r, const float* S, const float* V, const float* dS, const float* dV,
                      float eps_rel, float* K, cudaStream_t st) {
-  const size_t smem = (size_t)(2 * D * r + 2 * r * (r + 1) + D * (r + 1) + 2 * r) * sizeof(float);
+  const size_t smem = (size_t)(3 * D * (r | 1) + 2 * r * (r | 1) + 2 * r) * sizeof(float);
   cudaError_t e = cudaFuncSetAttribute(svd_grad_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   svd_grad_kernel<D><<<B, kGradThreads, smem, st>>>(S, V, dS, dV, eps_rel, r, K);
