@@ -21,6 +21,8 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
+constexpr int kUserThreads = 1024;   // the per-user chain is latency-bound: many warps per scheduler
+constexpr int kUserWarps = kUserThreads / 32;
 constexpr int kBatch = 32;            // candidate rows per inner batch
 constexpr int kRP = kTokenSlots;      // 64 token slots, zero padded
 
@@ -154,11 +156,45 @@ attn_bwd_rows_kernel(const T* __restrict__ C, const T* __restrict__ dO, T* __res
   }
 }
 
+// out(m, n) = sum_k a(m, k) b(k, n) for m < rows (rounded up to 4), n < D, by the whole CTA:
+// a warp takes four rows at a time, its lanes run along n with D/32 columns each, so one
+// step of k costs 4 broadcast reads of a and D/32 reads of b for 4*D/32 FMAs (the plain
+// one-output-per-thread loop is bound by shared-memory issue, not by the FMAs).
+template <int D, typename FA, typename FB, typename FS>
+__device__ __forceinline__ void small_gemm(int rows, int K, FA a, FB b, FS store, int warp, int lane,
+                                           int nwarps) {
+  constexpr int NC = D / 32;
+  for (int m0 = warp * 4; m0 < rows; m0 += nwarps * 4) {
+    float acc[4][NC];
+#pragma unroll
+    for (int x = 0; x < 4; ++x)
+#pragma unroll
+      for (int c = 0; c < NC; ++c) acc[x][c] = 0.f;
+#pragma unroll 4
+    for (int k = 0; k < K; ++k) {
+      float av[4], bv[NC];
+#pragma unroll
+      for (int x = 0; x < 4; ++x) av[x] = a(m0 + x, k);
+#pragma unroll
+      for (int c = 0; c < NC; ++c) bv[c] = b(k, lane + 32 * c);
+#pragma unroll
+      for (int x = 0; x < 4; ++x)
+#pragma unroll
+        for (int c = 0; c < NC; ++c) acc[x][c] = fmaf(av[x], bv[c], acc[x][c]);
+    }
+#pragma unroll
+    for (int x = 0; x < 4; ++x)
+#pragma unroll
+      for (int c = 0; c < NC; ++c)
+        if (m0 + x < rows) store(m0 + x, lane + 32 * c, acc[x][c]);
+  }
+}
+
 // Per-user chain from dT and dValue_r to dSigma, dV and this user's dW contributions.
 // Each weight matrix is staged in shared memory (fp32, odd pitch) when it is needed: W_K for
 // Key_r, W_Q for dKey_r, then W_K and W_V again for dA, where they are read along their rows.
 template <typename T, int D>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kUserThreads)
 attn_bwd_user_kernel(const float* __restrict__ part, int chunks, const float* __restrict__ S,
                      const float* __restrict__ V, const T* __restrict__ Wq, const T* __restrict__ Wk,
                      const T* __restrict__ Wv, float scale, int r, float* __restrict__ dS,
@@ -168,14 +204,14 @@ attn_bwd_user_kernel(const float* __restrict__ part, int chunks, const float* __
   constexpr int LW = D + 1;             // odd pitch of the staged weight matrix
   float* dT = sm;                       // [D][LR]    dT[k][i]
   float* dVT = dT + D * LR;             // [D][LR]    dValue_r^T[j][i]
-  float* A = dVT + D * LR;              // [kRP][D]   Sigma V^T, at the end dA
-  float* X = A + kRP * D;               // [kRP][D]   Key_r, then dKey_r
+  float* A = dVT + D * LR;              // [kRP][D]   Sigma V^T (rows past r zero), at the end dA
+  float* X = A + kRP * D;               // [kRP][D]   Key_r, then dKey_r (rows past r zero)
   float* Ws = X + kRP * D;              // [D][LW]    the weight matrix in use
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
   auto stage = [&](const T* __restrict__ W) {
     constexpr int VE = Vec16<T>::kElems;
-    for (int v = tid; v < D * D / VE; v += kThreads) {
+    for (int v = tid; v < D * D / VE; v += kUserThreads) {
       float tmp[VE];
       Vec16<T>::load(W + (size_t)v * VE, tmp);
       const int k = (v * VE) / D, j = (v * VE) % D;
@@ -186,98 +222,56 @@ attn_bwd_user_kernel(const float* __restrict__ part, int chunks, const float* __
 
   stage(Wk);
   // the partials, summed into the first chunk's slot by sum_chunks_kernel
-  for (int e = tid; e < 2 * D * kRP; e += kThreads)
+  for (int e = tid; e < 2 * D * kRP; e += kUserThreads)
     dT[(e / kRP) * LR + e % kRP] = part[(size_t)b * chunks * 2 * D * kRP + e];   // dVT follows dT in shared memory
-  for (int e = tid; e < kRP * D; e += kThreads) {
+  for (int e = tid; e < kRP * D; e += kUserThreads) {
     const int k = e / kRP, i = e % kRP;   // V is read along its rows
     A[i * D + k] = i < r ? S[(size_t)b * r + i] * V[((size_t)b * D + k) * r + i] : 0.f;
+    X[e] = 0.f;
   }
   __syncthreads();
-  // Key_r[i][j] = sum_k A[i][k] W_K[k][j]; lanes run over j
-  for (int e = tid; e < r * D; e += kThreads) {
-    const int i = e / D, j = e % D;
-    float acc = 0.f;
-#pragma unroll 8
-    for (int k = 0; k < D; ++k) acc = fmaf(A[i * D + k], Ws[k * LW + j], acc);
-    X[e] = acc;
-  }
+  // Key_r[i][j] = sum_k A[i][k] W_K[k][j]
+  small_gemm<D>(r, D, [&](int i, int k) { return A[i * D + k]; }, [&](int k, int j) { return Ws[k * LW + j]; },
+                [&](int i, int j, float v) { X[i * D + j] = v; }, warp, lane, kUserWarps);
   __syncthreads();
   stage(Wq);
   float* dWq = dw + (size_t)b * 3 * D * D;
   float* dWk = dWq + D * D;
   float* dWv = dWk + D * D;
   // dW_Q[k][j] = scale sum_i dT[k][i] Key_r[i][j]
-  for (int e = tid; e < D * D; e += kThreads) {
-    const int k = e / D, j = e % D;
-    float acc = 0.f;
-#pragma unroll 4
-    for (int i = 0; i < r; ++i) acc = fmaf(dT[k * LR + i], X[i * D + j], acc);
-    dWq[e] = scale * acc;
-  }
+  small_gemm<D>(D, r, [&](int k, int i) { return dT[k * LR + i]; }, [&](int i, int j) { return X[i * D + j]; },
+                [&](int k, int j, float v) { dWq[k * D + j] = scale * v; }, warp, lane, kUserWarps);
   __syncthreads();
   // dKey_r[i][j] = scale sum_k dT[k][i] W_Q[k][j]   (over Key_r)
-  for (int e = tid; e < r * D; e += kThreads) {
-    const int i = e / D, j = e % D;
-    float acc = 0.f;
-#pragma unroll 8
-    for (int k = 0; k < D; ++k) acc = fmaf(dT[k * LR + i], Ws[k * LW + j], acc);
-    X[e] = scale * acc;
-  }
+  small_gemm<D>(r, D, [&](int i, int k) { return dT[k * LR + i]; }, [&](int k, int j) { return Ws[k * LW + j]; },
+                [&](int i, int j, float v) { X[i * D + j] = scale * v; }, warp, lane, kUserWarps);
   __syncthreads();
   stage(Wk);
   // dW_K[k][j] = sum_i A[i][k] dKey_r[i][j],  dW_V[k][j] = sum_i A[i][k] dValue_r[i][j]
-  for (int e = tid; e < D * D; e += kThreads) {
-    const int k = e / D, j = e % D;
-    float ak = 0.f, av = 0.f;
-#pragma unroll 4
-    for (int i = 0; i < r; ++i) {
-      const float a = A[i * D + k];
-      ak = fmaf(a, X[i * D + j], ak);
-      av = fmaf(a, dVT[j * LR + i], av);
-    }
-    dWk[e] = ak;
-    dWv[e] = av;
-  }
+  small_gemm<D>(D, r, [&](int k, int i) { return A[i * D + k]; }, [&](int i, int j) { return X[i * D + j]; },
+                [&](int k, int j, float v) { dWk[k * D + j] = v; }, warp, lane, kUserWarps);
+  small_gemm<D>(D, r, [&](int k, int i) { return A[i * D + k]; }, [&](int i, int j) { return dVT[j * LR + i]; },
+                [&](int k, int j, float v) { dWv[k * D + j] = v; }, warp, lane, kUserWarps);
   __syncthreads();
-  // dA[i][k] = sum_j dKey_r[i][j] W_K[k][j] + dValue_r[i][j] W_V[k][j]; lanes run over k.
-  // Each thread keeps its entries in registers across the two staged matrices; dA then
-  // takes the place of A.
-  constexpr int QA = kRP * D / kThreads;
-  float acc_a[QA];
-#pragma unroll
-  for (int q = 0; q < QA; ++q) {
-    const int e = tid + q * kThreads, i = e / D, k = e % D;
-    float acc = 0.f;
-    if (i < r) {
-#pragma unroll 8
-      for (int j = 0; j < D; ++j) acc = fmaf(X[i * D + j], Ws[k * LW + j], acc);
-    }
-    acc_a[q] = acc;
-  }
+  // dA[i][k] = sum_j dKey_r[i][j] W_K[k][j] + dValue_r[i][j] W_V[k][j]; dA takes the place of A
+  small_gemm<D>(r, D, [&](int i, int j) { return X[i * D + j]; }, [&](int j, int k) { return Ws[k * LW + j]; },
+                [&](int i, int k, float v) { A[i * D + k] = v; }, warp, lane, kUserWarps);
   __syncthreads();
   stage(Wv);
   __syncthreads();
-#pragma unroll
-  for (int q = 0; q < QA; ++q) {
-    const int e = tid + q * kThreads, i = e / D, k = e % D;
-    float acc = acc_a[q];
-    if (i < r) {
-#pragma unroll 8
-      for (int j = 0; j < D; ++j) acc = fmaf(dVT[j * LR + i], Ws[k * LW + j], acc);
-    }
-    A[e] = acc;
-  }
+  small_gemm<D>(r, D, [&](int i, int j) { return dVT[j * LR + i]; }, [&](int j, int k) { return Ws[k * LW + j]; },
+                [&](int i, int k, float v) { A[i * D + k] += v; }, warp, lane, kUserWarps);
   __syncthreads();
   const float* dA = A;
   // dSigma_i = sum_k dA[i][k] V[k][i],  dV[k][i] = dA[i][k] sigma_i
-  for (int i = warp; i < r; i += kWarps) {
+  for (int i = warp; i < r; i += kUserWarps) {
     float acc = 0.f;
     for (int k = lane; k < D; k += 32) acc = fmaf(dA[i * D + k], V[((size_t)b * D + k) * r + i], acc);
 #pragma unroll
     for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
     if (lane == 0) dS[(size_t)b * r + i] = acc;
   }
-  for (int e = tid; e < D * r; e += kThreads) {
+  for (int e = tid; e < D * r; e += kUserThreads) {
     const int k = e / r, i = e % r;
     dV[(size_t)b * D * r + e] = dA[i * D + k] * S[(size_t)b * r + i];
   }
@@ -341,7 +335,7 @@ cudaError_t launch_td(int B, int M, int r, const void* C, const void* dO, const 
   const size_t smem_user = (size_t)(2 * D * (kRP + 1) + 2 * kRP * D + D * (D + 1)) * sizeof(float);
   e = cudaFuncSetAttribute(attn_bwd_user_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_user);
   if (e != cudaSuccess) return e;
-  attn_bwd_user_kernel<T, D><<<B, kThreads, smem_user, st>>>(part, chunks, S, V, static_cast<const T*>(Wq),
+  attn_bwd_user_kernel<T, D><<<B, kUserThreads, smem_user, st>>>(part, chunks, S, V, static_cast<const T*>(Wq),
                                                             static_cast<const T*>(Wk), static_cast<const T*>(Wv),
                                                             scale, r, dS, dV, dw);
   e = cudaGetLastError();

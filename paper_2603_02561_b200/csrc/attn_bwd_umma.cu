@@ -364,13 +364,13 @@ attn_bwd_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_const
 // Vkm [2][64][d] (Value_r, zero rows past r), each as a high and a low half.
 __global__ void attn_bwd_pack_kernel(const char* __restrict__ ws, AttnWs lay, int d, int r,
                                      __nv_bfloat16* __restrict__ pk) {
-  const int b = blockIdx.x;
+  const int b = blockIdx.y;
   const char* wsb = ws + (size_t)b * lay.per_user;
   const float* Tf = reinterpret_cast<const float*>(wsb + lay.tf_off);
   const float* Vr = reinterpret_cast<const float*>(wsb + lay.vr_off);
   __nv_bfloat16* Tkm = pk + (size_t)b * 4 * kTokenSlots * d;
   __nv_bfloat16* Vkm = Tkm + 2 * kTokenSlots * d;
-  for (int e = threadIdx.x; e < d * kTokenSlots; e += blockDim.x) {
+  for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < d * kTokenSlots; e += gridDim.x * blockDim.x) {
     const int k = e / kTokenSlots, i = e % kTokenSlots;
     const float t = i < r ? Tf[k * r + i] : 0.f;
     const __nv_bfloat16 th = __float2bfloat16_rn(t);
@@ -389,7 +389,7 @@ cudaError_t launch_d(int B, int M, int r, const void* C, const void* dO, unsigne
                      __nv_bfloat16* pk, int tiles_per_cta, int chunks, const char* ws, const AttnWs& lay,
                      cudaStream_t st) {
   using Cfg = BwdCfg<D>;
-  attn_bwd_pack_kernel<<<B, 256, 0, st>>>(ws, lay, D, r, pk);
+  attn_bwd_pack_kernel<<<dim3(D * kTokenSlots / 256, B), 256, 0, st>>>(ws, lay, D, r, pk);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   CUtensorMap tmC, tmG, tmDC, tmT, tmVk, tmTk;

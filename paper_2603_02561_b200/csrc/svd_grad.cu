@@ -22,7 +22,7 @@ namespace solar {
 
 namespace {
 
-constexpr int kGradThreads = 256;
+constexpr int kGradThreads = 1024;   // latency-bound small products: many warps per scheduler
 
 template <int D>
 __global__ void __launch_bounds__(kGradThreads)
