@@ -422,6 +422,44 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
                     "roofline": {"bound": "alu", "achieved": exps / (f_ms * 1e-3) / 1e12, "peak": SFU_TEXPS,
                                  "unit": "Texp/s", "frac": exps / (f_ms * 1e-3) / 1e12 / SFU_TEXPS,
                                  "note": "one exp2 per candidate x position on the special-function units"}}
+    # the backward pass (beside the hot path, not part of `value`): attention part, then the
+    # SVD's gradient as one more streaming pass over H; graph replay over the same batches
+    backward = None
+    if not light:
+        bws = solar.alloc_backward_workspace(w.B, w.M, w.N, w.d, w.r, tdt)
+        dHg = torch.empty_like(dH[0])
+        gO = [torch.randn(w.B, w.M, w.d, device="cuda").to(tdt) for _ in range(nb)]
+        grads = solar.alloc_attention_grads(dC[0], w.r)
+
+        def bwd_part(k, which):
+            if which in (0, 2):
+                solar.svd_attention_bwd(dC[k], lane0.S, lane0.V, Wq, Wk, Wv, w.scale, gO[k], bws, out=grads,
+                                        stream=main_stream)
+            if which in (1, 2):
+                solar.svd_backward(dH[k], lane0.S, lane0.V, grads[4], grads[5], dHg, bws, stream=main_stream)
+
+        with torch.cuda.stream(main_stream):
+            solar.lowrank_factor(dH[0], w.r, S=lane0.S, V=lane0.V, workspace=lane0.ws, M=w.M, stream=main_stream)
+            bwd_part(0, 2)
+        torch.cuda.synchronize()
+        b_ms = []
+        for which in (0, 1, 2):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(main_stream):
+                with torch.cuda.graph(g, stream=main_stream, capture_error_mode="relaxed"):
+                    for k in range(nb):
+                        bwd_part(k, which)
+                g.replay()
+            torch.cuda.synchronize()
+            a, b = timed_replays(g, 5)
+            torch.cuda.synchronize()
+            b_ms.append(a.elapsed_time(b) / (5 * nb))
+        es = 2 if w.dtype == "bf16" else 4
+        bwd_bytes = es * w.B * (3 * w.M * w.d + 2 * w.N * w.d)        # C, dO, dC; H, dH
+        backward = {"ms_per_call": b_ms[2], "attention_bwd_ms": b_ms[0], "svd_backward_ms": b_ms[1],
+                    "what": "solar_svd_attention_bwd + solar_svd_backward, one batch at a time on one stream",
+                    "roofline": {"bound": "hbm", "achieved": bwd_bytes / (b_ms[2] * 1e-3) / 1e9,
+                                 "unit": "GB/s", "algorithmic_bytes": bwd_bytes}}
     clocks = sampler.stop() if rank == 0 else None
 
     # end to end through the public API with host buffers (pinned), copies inside the timed region
@@ -497,6 +535,7 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
         "gpu_launches": KERNELS_PER_STEP * steps,
         "clocks": clocks,
         "factored_exact": factored,
+        "backward": backward,
         "e2e": {"value": world * w.pairs * e2e_steps / e2e_s, "unit": "pairs/s",
                 "h2d_bytes_per_step": hH.numel() * hH.element_size() + hC.numel() * hC.element_size(),
                 "d2h_bytes_per_step": hO.numel() * hO.element_size(), "steps": e2e_steps},

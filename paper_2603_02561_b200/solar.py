@@ -233,17 +233,24 @@ def alloc_backward_workspace(B, M, N, d, r, dtype, device="cuda") -> torch.Tenso
     return torch.empty(max(backward_workspace_bytes(B, M, N, d, r, dtype), 256), dtype=torch.uint8, device=device)
 
 
-def svd_attention_bwd(C, S, V, Wq, Wk, Wv, scale, dO, workspace, flags=0, stream=None):
+def alloc_attention_grads(C, r):
+    """Output tensors of svd_attention_bwd: dC, dWq, dWk, dWv, dS, dV."""
+    B, M, d = C.shape
+    dev = C.device
+    return (torch.empty_like(C), *(torch.empty(d, d, dtype=torch.float32, device=dev) for _ in range(3)),
+            torch.empty(B, r, dtype=torch.float32, device=dev), torch.empty(B, d, r, dtype=torch.float32, device=dev))
+
+
+def svd_attention_bwd(C, S, V, Wq, Wk, Wv, scale, dO, workspace, flags=0, out=None, stream=None):
     """solar_svd_attention_bwd: gradients of the forward call's inputs given dO.
-    Returns dC[B,M,d], dWq, dWk, dWv [d,d] f32, dS[B,r], dV[B,d,r]."""
+    Returns dC[B,M,d], dWq, dWk, dWv [d,d] f32, dS[B,r], dV[B,d,r] (written into `out` if given)."""
     B, M, d = C.shape
     r = S.shape[1]
     _need(dO, (B, M, d), C.dtype, "dO")
-    dev = C.device
-    dC = torch.empty_like(C)
-    dWq, dWk, dWv = (torch.empty(d, d, dtype=torch.float32, device=dev) for _ in range(3))
-    dS = torch.empty(B, r, dtype=torch.float32, device=dev)
-    dV = torch.empty(B, d, r, dtype=torch.float32, device=dev)
+    dC, dWq, dWk, dWv, dS, dV = alloc_attention_grads(C, r) if out is None else out
+    _need(dC, (B, M, d), C.dtype, "dC"); _need(dS, (B, r), torch.float32, "dS"); _need(dV, (B, d, r), torch.float32, "dV")
+    for nm, W in (("dWq", dWq), ("dWk", dWk), ("dWv", dWv)):
+        _need(W, (d, d), torch.float32, nm)
     _check(lib().solar_svd_attention_bwd(B, M, max(r, 1), d, r, dtype_code(C.dtype), _ptr(C), _ptr(S), _ptr(V),
                                          _ptr(Wq), _ptr(Wk), _ptr(Wv), float(scale), int(flags), _ptr(dO),
                                          _ptr(dC), _ptr(dWq), _ptr(dWk), _ptr(dWv), _ptr(dS), _ptr(dV),
