@@ -43,10 +43,10 @@ SFU_TEXPS = 148 * 16 * 1.965e9 / 1e12              # 148 SMs x 16 special-functi
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (null once the kernel has changed since the capture)
 TRAFFIC = {
-    ("c3", "gram"): 20988160,        # profiles/gram_umma_c3.md
+    ("c3", "gram"): 20987904,        # profiles/gram_umma_c3.md
     ("c3", "attn_apply"): 4628224,   # profiles/attn_umma_c3.md (O still in L2 when the kernel ends)
-    ("c3", "eig"): 2430464,          # profiles/eig_kernel_c3.md
-    ("c3", "attn_prepare"): 183040,  # profiles/attn_prepare_c3.md
+    ("c3", "eig"): 2432000,          # profiles/eig_kernel_c3.md
+    ("c3", "attn_prepare"): 187136,  # profiles/attn_prepare_c3.md
 }
 
 

@@ -446,17 +446,19 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
   for (int s = tid; s < splits; s += NT) lost |= (gram_status[b * splits + s] != kGramStatusOk);
   int bad = 0;
   for (int e = tid; e < D * D / 4; e += NT) {
-    // fp32 sums in a fixed order (eight slices at a time, pairwise within the eight): the
-    // partials are fp32 to begin with, and one rounding per level is far below their own error
+    // fp32 sums in a fixed order (GW slices at a time, pairwise within the group): the
+    // partials are fp32 to begin with, and one rounding per level is far below their own error.
+    // All loads of a group are issued before the first add: the loop is bound by their latency.
+    constexpr int GW = (D == 128) ? 8 : 16;      // 1024 threads leave 64 registers each at d = 128
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s = 0; s < splits; s += 8) {
-      float4 v[8];
+    for (int s = 0; s < splits; s += GW) {
+      float4 v[GW];
 #pragma unroll
-      for (int u = 0; u < 8; ++u)
+      for (int u = 0; u < GW; ++u)
         v[u] = (s + u < splits) ? __ldg(gp + (size_t)(s + u) * (D * D / 4) + e)
                                 : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-      for (int h = 4; h >= 1; h >>= 1)
+      for (int h = GW / 2; h >= 1; h >>= 1)
 #pragma unroll
         for (int u = 0; u < h; ++u) {
           v[u].x += v[u + h].x; v[u].y += v[u + h].y; v[u].z += v[u + h].z; v[u].w += v[u + h].w;

@@ -201,7 +201,7 @@ solar_status_t solar_svd_attention_bwd(int B, int M, int N, int d, int r, solar_
                                        void* workspace, size_t workspace_bytes, void* stream) {
   (void)N;
   SOLAR_TRY(check_dims(B, M, r, d, r, dt));
-  if (flags & ~(unsigned)SOLAR_FLAG_NO_SOFTMAX) return SOLAR_ERR_INVALID_ARG;
+  if (flags & ~(unsigned)SOLAR_FLAG_NO_SOFTMAX) return SOLAR_ERR_UNSUPPORTED;
   if (B == 0) return SOLAR_OK;
   if (M > 0) { SOLAR_TRY(check_ptr(C)); SOLAR_TRY(check_ptr(dO)); SOLAR_TRY(check_ptr(dC)); }
   SOLAR_TRY(check_ptr(S));

@@ -77,6 +77,38 @@ def test_host_side_rejections_need_no_gpu(L):
     assert st == solar.ERR_WORKSPACE
 
 
+def test_backward_calls_reject_bad_arguments_on_the_host(L):
+    vp = ctypes.c_void_p
+    p = vp(0x1000)
+    bf = torch.bfloat16
+    need = solar.backward_workspace_bytes(16, 2048, 10240, 64, 32, bf)
+    # attention workspace, per-chunk partials [B][chunks][2][d][64] f32, dW [B][3][d][d] f32, operands
+    assert need >= solar.workspace_bytes(16, 2048, 32, 64, 32, bf) // 2
+    assert need >= 16 * 2 * 64 * 64 * 4 + 16 * 3 * 64 * 64 * 4
+    assert need >= 16 * 64 * 64 * 4                                         # K_b of solar_svd_backward
+    assert solar.backward_workspace_bytes(1, 16, 256, 48, 8, bf) == 0       # unsupported d
+
+    def bwd(B=1, M=4, d=64, r=8, dt=1, flags=0, wsb=1 << 40, C=p):
+        return L.solar_svd_attention_bwd(B, M, 256, d, r, dt, C, p, p, p, p, p, 0.125, flags, p,
+                                         p, p, p, p, p, p, p, wsb, None)
+    assert bwd(d=48) == solar.ERR_UNSUPPORTED
+    assert bwd(r=65) == solar.ERR_INVALID_ARG
+    assert bwd(flags=2) == solar.ERR_UNSUPPORTED
+    assert bwd(wsb=64) == solar.ERR_WORKSPACE
+    assert bwd(C=vp(0)) == solar.ERR_INVALID_ARG
+    assert bwd(B=0) == solar.OK
+
+    def svdb(B=1, N=256, d=64, r=8, eps=0.0, wsb=1 << 40, H=p):
+        return L.solar_svd_backward(B, N, d, r, 1, H, p, p, p, p, eps, p, p, wsb, None)
+    assert svdb(d=48) == solar.ERR_UNSUPPORTED
+    assert svdb(N=4) == solar.ERR_INVALID_ARG                               # r > N
+    assert svdb(eps=-1.0) == solar.ERR_INVALID_ARG
+    assert svdb(eps=float("nan")) == solar.ERR_INVALID_ARG
+    assert svdb(wsb=64) == solar.ERR_WORKSPACE
+    assert svdb(H=vp(0x1002)) == solar.ERR_INVALID_ARG
+    assert svdb(B=0) == solar.OK
+
+
 def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
     monkeypatch.setattr(solar, "_lib", None)
     monkeypatch.setattr(solar, "LIB_PATH", str(tmp_path / "missing.so"))

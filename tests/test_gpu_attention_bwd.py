@@ -106,4 +106,4 @@ def test_attention_bwd_argument_checks():
     assert e.value.status == solar.ERR_WORKSPACE
     with pytest.raises(solar.SolarError) as e:
         solar.svd_attention_bwd(C, S, V, Wq, Wk, Wv, inp["scale"], dO, bws, flags=2)
-    assert e.value.status == solar.ERR_INVALID_ARG
+    assert e.value.status == solar.ERR_UNSUPPORTED
