@@ -48,6 +48,17 @@ def _rel(got, ref):
     return np.abs(got - ref).max() / max(np.abs(ref).max(), 1e-300)
 
 
+def _check_dC(got, ref, dtype):
+    """dC against the oracle.  A row of dC = dS T^T is a difference of terms (dS = P o (dP - rowsum));
+    where the softmax saturates the row nearly cancels, so the error is measured against the
+    matrix's scale, and row by row only on the rows that carry weight."""
+    tol = 2.0 ** -7 if dtype == "bf16" else 1e-4          # one rounding to the storage type
+    assert _rel(got, ref) <= tol
+    rows = np.abs(ref).max(axis=1) >= 1e-2 * np.abs(ref).max()
+    assert rows.any()
+    assert o.max_rel_err_rows(got[rows], ref[rows]) <= (2e-2 if dtype == "bf16" else 1e-4)
+
+
 @pytest.mark.parametrize("w,flags", CASES, ids=[f"{c[0].name}_M{c[0].M}_r{c[0].r}_f{c[1]}" for c in CASES])
 def test_attention_bwd_matches_oracle(w, flags):
     inp, H, C, Wq, Wk, Wv, S, V, dO, bws = _setup(w, seed=w.M + w.r)
@@ -57,12 +68,11 @@ def test_attention_bwd_matches_oracle(w, flags):
     S64, V64, dO64 = _f64(S), _f64(V), _f64(dO)
     B = S64.shape[0]
     sums = {k: 0.0 for k in ("dWq", "dWk", "dWv")}
-    out_tol = 1e-2 if w.dtype == "bf16" else 1e-4       # dC is rounded to the storage type
     for k in range(B):
         g = ob.svd_attention_backward(inp["C"][k].astype(np.float64), S64[k], V64[k],
                                       *(inp[n].astype(np.float64) for n in ("Wq", "Wk", "Wv")),
                                       inp["scale"], dO64[k], softmax=not flags)
-        assert o.max_rel_err_rows(_f64(dC[k]), g["dC"]) <= out_tol
+        _check_dC(_f64(dC[k]), g["dC"], w.dtype)
         assert _rel(_f64(dS[k]), g["ds"]) <= 1e-4
         assert _rel(_f64(dV[k]), g["dV"]) <= 1e-4
         for n in sums:
@@ -84,6 +94,36 @@ def test_whole_backward_pass_matches_oracle():
                                            S64[k], V64[k], *(inp[n].astype(np.float64) for n in ("Wq", "Wk", "Wv")),
                                            inp["scale"], dO64[k])
         assert _rel(_f64(dH[k]), g["dH"]) <= 2.0 ** -7
+
+
+@pytest.mark.parametrize("name,users", [("c3", (0, 15)), ("c4", (3,))])
+def test_full_size_backward_sampled_users(name, users):
+    """The headline shapes in the launch configuration the benchmark times: every gradient of the
+    sampled users against the oracle (dW sums need all users: checked through per-user partial sums
+    of the oracle over ALL users for c3 only, where that is cheap)."""
+    w = wl.CONFIGS[name]
+    inp, H, C, Wq, Wk, Wv, S, V, dO, bws = _setup(w, seed=17)
+    dC, dWq, dWk, dWv, dS, dV = solar.svd_attention_bwd(C, S, V, Wq, Wk, Wv, inp["scale"], dO, bws)
+    dH = torch.empty_like(H)
+    solar.svd_backward(H, S, V, dS, dV, dH, bws, eps_rel=1e-4)
+    torch.cuda.synchronize()
+    S64, V64, dO64 = _f64(S), _f64(V), _f64(dO)
+    W64 = [inp[n].astype(np.float64) for n in ("Wq", "Wk", "Wv")]
+    sums = {k: 0.0 for k in ("dWq", "dWk", "dWv")}
+    for k in (range(w.B) if name == "c3" else users):
+        g = ob.svd_attention_backward(inp["C"][k].astype(np.float64), S64[k], V64[k], *W64, inp["scale"], dO64[k])
+        for n in sums:
+            sums[n] = sums[n] + g[n]
+        if k not in users:
+            continue
+        _check_dC(_f64(dC[k]), g["dC"], w.dtype)
+        assert _rel(_f64(dS[k]), g["ds"]) <= 1e-4
+        assert _rel(_f64(dV[k]), g["dV"]) <= 1e-4
+        ref = ob.svd_backward(inp["H"][k].astype(np.float64), S64[k], V64[k], _f64(dS[k]), _f64(dV[k]), 1e-4)
+        assert _rel(_f64(dH[k]), ref) <= 2.0 ** -7
+    if name == "c3":
+        for n, t in (("dWq", dWq), ("dWk", dWk), ("dWv", dWv)):
+            assert _rel(_f64(t), sums[n]) <= 1e-4, n
 
 
 def test_attention_bwd_is_reproducible_bit_for_bit():
