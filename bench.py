@@ -459,7 +459,10 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
         backward = {"ms_per_call": b_ms[2], "attention_bwd_ms": b_ms[0], "svd_backward_ms": b_ms[1],
                     "what": "solar_svd_attention_bwd + solar_svd_backward, one batch at a time on one stream",
                     "roofline": {"bound": "hbm", "achieved": bwd_bytes / (b_ms[2] * 1e-3) / 1e9,
-                                 "unit": "GB/s", "algorithmic_bytes": bwd_bytes}}
+                                 "peak": peaks()["hbm_gbs"], "unit": "GB/s",
+                                 "frac": bwd_bytes / (b_ms[2] * 1e-3) / 1e9 / peaks()["hbm_gbs"],
+                                 "algorithmic_bytes": bwd_bytes,
+                                 "note": "eight short kernels back to back: latency- and launch-bound"}}
     clocks = sampler.stop() if rank == 0 else None
 
     # end to end through the public API with host buffers (pinned), copies inside the timed region

@@ -138,6 +138,39 @@ def test_attention_bwd_is_reproducible_bit_for_bit():
         assert torch.equal(x.view(torch.uint8), y.view(torch.uint8))
 
 
+def test_no_candidates_gives_zero_gradients():
+    w = wl.CONFIGS["c2"].with_(B=2, M=1)
+    inp, H, C, Wq, Wk, Wv, S, V, dO, bws = _setup(w, seed=2)
+    C0, dO0 = C[:, :0, :].contiguous(), dO[:, :0, :].contiguous()
+    dC, dWq, dWk, dWv, dS, dV = solar.svd_attention_bwd(C0, S, V, Wq, Wk, Wv, inp["scale"], dO0, bws)
+    torch.cuda.synchronize()
+    for t in (dWq, dWk, dWv, dS, dV):
+        assert torch.count_nonzero(t) == 0 and torch.isfinite(t).all()
+
+
+def test_zero_history_has_zero_gradient_and_no_nan():
+    """H = 0: every sigma is zero, so no direction has a U column and dH = 0 (no 0/0)."""
+    B, N, d, r, M = 2, 300, 64, 8, 40
+    H = torch.zeros(B, N, d, dtype=torch.bfloat16, device="cuda")
+    g = torch.Generator().manual_seed(9)
+    C = (torch.randn(B, M, d, generator=g) / 8).to(torch.bfloat16).cuda()
+    dO = torch.randn(B, M, d, generator=g).to(torch.bfloat16).cuda()
+    Wq, Wk, Wv = ((torch.randn(d, d, generator=g) / 8).to(torch.bfloat16).cuda() for _ in range(3))
+    ws = solar.alloc_workspace(B, M, N, d, r, torch.bfloat16)
+    S, V = solar.lowrank_factor(H, r, workspace=ws)
+    bws = solar.alloc_backward_workspace(B, M, N, d, r, torch.bfloat16)
+    out = solar.svd_attention_bwd(C, S, V, Wq, Wk, Wv, 0.125, dO, bws)
+    dH = torch.full_like(H, float("nan"))
+    solar.svd_backward(H, S, V, out[4], out[5], dH, bws)
+    torch.cuda.synchronize()
+    assert torch.count_nonzero(S) == 0
+    for t in out:
+        assert torch.isfinite(t.float()).all()
+    assert torch.count_nonzero(dH) == 0
+    # scores are all zero, so the probabilities are uniform and dC vanishes with T = 0
+    assert torch.count_nonzero(out[0]) == 0
+
+
 def test_attention_bwd_argument_checks():
     w = wl.CONFIGS["c1"]
     inp, H, C, Wq, Wk, Wv, S, V, dO, bws = _setup(w, seed=1)
