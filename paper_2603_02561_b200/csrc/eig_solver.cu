@@ -712,6 +712,7 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
     float* Wc = Vm;                                  // [D cols][D rows]
     int* perm = order + D;                           // [2][D]
     const int I = tid % HP, Jb = tid / HP;
+    static_assert(HP == 16 || HP == 32 || HP == 64, "rotation sharing by shuffle");
 
     float xin[PTJ][4];
 #pragma unroll
@@ -746,13 +747,30 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
         const float* Tc = cur ? Gn : Gc;
         float* Tn = cur ? Gc : Gn;
         const int* pc = perm + cur * D;
-        bool big_r, big_c;
-        const Rot rr = jacobi_rot(Tc[srcI], Tc[3 * PLN + srcI], Tc[PLN + srcI], thr_abs2, stop2, big_r);
+        // The lanes of every warp compute the round's HP rotations between them (lane l takes
+        // the pairs l, l + 32, ...); a thread's row rotation is among its own, and the column
+        // rotations, uniform across the warp, come by shuffle -- instead of every thread
+        // computing one rotation per block it owns.
+        constexpr int NR = (HP + 31) / 32;
+        Rot rl[NR];
+#pragma unroll
+        for (int q = 0; q < NR; ++q) {
+          const int pr = (HP >= 32) ? q * 32 + lane : lane % HP;
+          const int sp = pr * (HP + 1) + pr;
+          bool big;
+          rl[q] = jacobi_rot(Tc[sp], Tc[3 * PLN + sp], Tc[PLN + sp], thr_abs2, stop2, big);
+          worst |= big;
+        }
+        Rot rr = rl[0];
+        if (NR == 2 && I >= 32) rr = rl[NR - 1];
 #pragma unroll
         for (int c = 0; c < PTJ; ++c) {
-          const int J = Jb + c * NJ, srcJ = J * (HP + 1) + J, src = I * (HP + 1) + J;
-          const Rot rc = jacobi_rot(Tc[srcJ], Tc[3 * PLN + srcJ], Tc[PLN + srcJ], thr_abs2, stop2, big_c);
-          worst |= big_c;
+          const int J = Jb + c * NJ, src = I * (HP + 1) + J;
+          const Rot& rs = (NR == 2 && J >= 32) ? rl[NR - 1] : rl[0];   // J is uniform across the warp
+          Rot rc;
+          rc.s = __shfl_sync(0xffffffffu, rs.s, J & 31);
+          rc.tau = __shfl_sync(0xffffffffu, rs.tau, J & 31);
+          rc.t = rr.t;                       // used only where I == J
           float x00 = Tc[src], x01 = Tc[PLN + src], x10 = Tc[2 * PLN + src], x11 = Tc[3 * PLN + src];
           float2* wa = reinterpret_cast<float2*>(Wc + pc[2 * J] * D + 2 * I);
           float2* wb = reinterpret_cast<float2*>(Wc + pc[2 * J + 1] * D + 2 * I);
