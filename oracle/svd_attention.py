@@ -11,7 +11,7 @@ d (embedding width), r (rank).  One user at a time; batches are Python loops.
 
 Pin status: every function below is pinned by tests/test_oracle_pins.py
 (closed forms, invariants, a LAPACK SVD, brute force, a hand-computed golden
-case).  Two conventions are this build's own and are "parity unpinned" against
+case).  Two conventions are this implementation's own and are "parity unpinned" against
 the authors' unpublished system: the sign gauge of V (`sign_gauge`) and the
 value of `scale` (an explicit argument; the paper prints no 1/sqrt(d)).
 """
@@ -83,7 +83,7 @@ def hestenes_svd(H, tol=1e-15, max_sweeps=60):
 def sign_gauge(V):
     """Fix the sign of each right singular vector (column of V[d,r]).
 
-    Convention of this build (the paper is silent and the softmax over the r
+    Convention of this implementation (the paper is silent and the softmax over the r
     factor-tokens is NOT invariant to v_i -> -v_i): the component of largest
     magnitude is made positive; ties go to the lowest index.  Returns
     (V_fixed, flips[r]) with flips in {+1,-1} such that V_fixed = V * flips.

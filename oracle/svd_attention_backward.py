@@ -24,7 +24,7 @@ that is Eq. 15 with the Hadamard factor Vbar^T V in place of V^T Vbar.  Finite d
 
 Stabilisation of F (the paper gives none): F_ij = D / (D^2 + eps^2) with
 D = sigma_i^2 - sigma_j^2 and eps = eps_rel * sigma_1^2; eps_rel = 0 is Eq. 14 itself
-(and F_ij = 0 where D = 0).  This convention is this build's own: "parity unpinned"
+(and F_ij = 0 where D = 0).  This convention is this implementation's own: "parity unpinned"
 against the authors' system for eps_rel > 0; for eps_rel = 0 everything here is pinned.
 """
 from __future__ import annotations
