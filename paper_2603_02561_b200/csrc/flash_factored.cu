@@ -231,16 +231,24 @@ flash_factored_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_cons
 #pragma unroll
       for (int j = 0; j < kPos; ++j) s[j] = (j < valid) ? s[j] : -INFINITY;
     }
-    float m_new = m_run;
+    // eight independent chains for the maximum and for the sum: with two warps per scheduler a
+    // 128-long dependent chain would be exposed latency
+    float mx[8], sm8[8];
 #pragma unroll
-    for (int j = 0; j < kPos; ++j) m_new = fmaxf(m_new, s[j]);
+    for (int q = 0; q < 8; ++q) mx[q] = s[q];
+#pragma unroll
+    for (int j = 8; j < kPos; ++j) mx[j & 7] = fmaxf(mx[j & 7], s[j]);
+    const float m_new = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
+                              fmaxf(fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])), m_run));
     const float alpha = ex2(m_run - m_new);         // 0 on the first tile (m_run = -inf)
-    float sum = 0.f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) sm8[q] = 0.f;
 #pragma unroll
     for (int j = 0; j < kPos; ++j) {
       s[j] = ex2(s[j] - m_new);                     // masked positions: 2^-inf = 0
-      sum += s[j];
+      sm8[j & 7] += s[j];
     }
+    const float sum = ((sm8[0] + sm8[1]) + (sm8[2] + sm8[3])) + ((sm8[4] + sm8[5]) + (sm8[6] + sm8[7]));
     l_run = fmaf(l_run, alpha, sum);
     m_run = m_new;
 #pragma unroll
