@@ -218,13 +218,19 @@ flash_factored_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_cons
 
     // this thread's 128 scores (already in log2 units): running max, exp2, running sum
     float s[kPos];
-#pragma unroll
-    for (int c = 0; c < kPos / 32; ++c) {
-      uint32_t v[32];
-      ptx::tmem_ld_32x32(tm_s + lane_base + c * 32, v);
+    {
+      // all four loads in flight, one wait
+      uint32_t v0[32], v1[32], v2[32], v3[32];
+      ptx::tmem_ld_32x32(tm_s + lane_base, v0);
+      ptx::tmem_ld_32x32(tm_s + lane_base + 32, v1);
+      ptx::tmem_ld_32x32(tm_s + lane_base + 64, v2);
+      ptx::tmem_ld_32x32(tm_s + lane_base + 96, v3);
       ptx::tmem_ld_wait();
 #pragma unroll
-      for (int i = 0; i < 32; ++i) s[c * 32 + i] = __uint_as_float(v[i]);
+      for (int i = 0; i < 32; ++i) {
+        s[i] = __uint_as_float(v0[i]);      s[32 + i] = __uint_as_float(v1[i]);
+        s[64 + i] = __uint_as_float(v2[i]); s[96 + i] = __uint_as_float(v3[i]);
+      }
     }
     const int valid = N - t * kPos;                 // positions past N hold zero-filled rows
     if (valid < kPos) {
