@@ -117,6 +117,26 @@ def test_truncated_case_inside_the_subspace():
     assert np.abs(U @ (U.T @ dH @ V) @ V.T - dH).max() < 1e-12 * max(1.0, np.abs(dH).max())
 
 
+def test_diagonal_2x2_against_first_order_perturbation_theory():
+    """H = diag(a, b), a > b > 0: U = V = I.  Textbook perturbation of the eigenvectors of H^T H:
+    adding eps at (1,2) turns v1 by +a eps/(a^2-b^2) towards e2 (and v2 by the opposite), adding
+    eps at (2,1) turns it by +b eps/(a^2-b^2).  So for a loss with dL/dV = R and dL/dSigma = g:
+      dL/dH = [[g1, a (R21 - R12)/(a^2-b^2)], [b (R21 - R12)/(a^2-b^2), g2]]."""
+    a, b = 3.0, 2.0
+    H = np.diag([a, b])
+    s, V = np.array([a, b]), np.eye(2)
+    R = np.array([[0.3, -1.1], [0.7, 0.4]])
+    g = np.array([0.5, -0.25])
+    k = (R[1, 0] - R[0, 1]) / (a * a - b * b)
+    want = np.array([[g[0], a * k], [b * k, g[1]]])
+    got = ob.svd_backward(H, s, V, g, R)
+    assert np.abs(got - want).max() < 1e-14
+    # the same numbers, worked by hand, in the golden file
+    import os
+    gold = np.loadtxt(os.path.join(os.path.dirname(__file__), "golden", "diag2x2_svd_backward.txt"))
+    assert np.abs(got - gold).max() < 1e-14
+
+
 def test_F_and_its_stabilisation():
     s = np.array([3.0, 2.0, 1.0])
     F = ob.svd_grad_F(s)
