@@ -151,7 +151,10 @@ def run_reference(args, w: wl.Workload):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    sample_users = list(range(min(w.B, args.ref_users)))
+    # a bounded sample per step: fewer users per step when many steps are asked for, so that the
+    # whole run stays within a few minutes of host time
+    per_step = args.ref_users if args.steps <= 8 else 1
+    sample_users = list(range(min(w.B, per_step)))
     for _ in range(min(args.warmup, 1)):
         oracle_step(w, sample_users[:1])
     ts = [oracle_step(w, sample_users) for _ in range(args.steps)]
