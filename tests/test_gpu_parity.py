@@ -82,6 +82,8 @@ SMALL = [
     ("f32", 3, 300, 32, 8, 65), ("f32", 2, 1000, 64, 64, 1), ("f32", 1, 257, 128, 33, 130),
     ("bf16", 3, 300, 32, 32, 65), ("bf16", 2, 1000, 64, 1, 7), ("bf16", 2, 515, 128, 64, 200),
     ("bf16", 5, 129, 64, 27, 64), ("f32", 2, 64, 64, 64, 3),
+    # subspace dimensions 24 and 16 of the range-finder route (Ritz problems of every layout)
+    ("bf16", 2, 700, 64, 20, 40), ("bf16", 2, 400, 128, 24, 50), ("f32", 2, 600, 128, 12, 33),
 ]
 
 
