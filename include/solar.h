@@ -55,20 +55,33 @@ enum {
 enum {
   SOLAR_INFO_NOT_CONVERGED = 1, /* sweep cap reached before every rotation became negligible */
   SOLAR_INFO_NONFINITE = 2,     /* H_b^T H_b contains NaN or Inf; s, V of this user are NaN  */
-  SOLAR_INFO_NOT_CERTIFIED = 4, /* only with SOLAR_ROUTE_SUBSPACE: the range-finder result was
-                                   written although its error bounds did not hold              */
+  SOLAR_INFO_NOT_CERTIFIED = 4, /* only with SOLAR_ROUTE_SUBSPACE / SOLAR_ROUTE_TRIDIAG: the result
+                                   was written although its error bounds did not hold          */
   SOLAR_INFO_DEVICE_WAIT = 8    /* a bounded wait inside the Gram kernel (on a TMA copy or on the
                                    tensor cores) ran out; s, V of this user are NaN             */
 };
 
 /* How solar_eig_from_partials_ex reaches the top-r eigenpairs of H_b^T H_b.
- * AUTO (what solar_lowrank_factor uses): Algorithm 1 (randomized range finder with
- * power iteration) applied to the d x d Gram matrix, accepted per user only when
- * residual and trace bounds certify the r pairs, else the full d x d Jacobi
- * eigensolver.  SUBSPACE: the range finder alone, uncertified users flagged in
- * info[].  FULL: the full eigensolver for every user (Eq. 9's exact truncated SVD
- * whatever the spectrum). */
-enum { SOLAR_ROUTE_AUTO = 0, SOLAR_ROUTE_SUBSPACE = 1, SOLAR_ROUTE_FULL = 2 };
+ * AUTO (what solar_lowrank_factor uses): Householder tridiagonalisation of the d x d
+ * matrix, the r largest eigenvalues by Sturm-count multisection, their vectors by the
+ * twisted factorisation, back-transformation; accepted per user only when the residuals
+ * G v - theta v against the Gram matrix itself, V^T V = I and the trace certify the r
+ * pairs, else the parallel Jacobi eigensolver on the whole matrix runs for that user.
+ * SUBSPACE: Algorithm 1 (randomized range finder with power iteration) applied to the
+ * d x d Gram matrix, then a Rayleigh-Ritz solve, alone; users whose residual and trace
+ * bounds do not certify the result are flagged in info[].  FULL: the Jacobi eigensolver for every user (Eq. 9's exact
+ * truncated SVD whatever the spectrum).  TRIDIAG: the tridiagonal route alone,
+ * uncertified users flagged in info[].
+ *
+ * The route argument may carry two more fields above the low byte (both 0 = default):
+ *   bits  8..15  sweep cap of the Jacobi eigensolver (1..16; default 16): a user not
+ *                converged by then gets SOLAR_INFO_NOT_CONVERGED;
+ *   bits 16..23  with SUBSPACE: run exactly this many orthonormalised power steps
+ *                (Algorithm 1 with n_iter = value - 1, value <= 5) instead of the adaptive
+ *                count. */
+enum { SOLAR_ROUTE_AUTO = 0, SOLAR_ROUTE_SUBSPACE = 1, SOLAR_ROUTE_FULL = 2, SOLAR_ROUTE_TRIDIAG = 3 };
+#define SOLAR_ROUTE_WITH(route, sweep_cap, power_steps) \
+  ((route) | ((sweep_cap) << 8) | ((power_steps) << 16))
 
 const char* solar_status_string(solar_status_t st);
 
@@ -90,10 +103,12 @@ size_t solar_workspace_bytes(int B, int M, int N, int d, int r, solar_dtype_t dt
  *   info [B] int      (out)  SOLAR_INFO_* bits per user, or NULL
  *
  * Route: G_b = H_b^T H_b is accumulated in one streaming pass over H; its top-r
- * eigenpairs come from Algorithm 1 (randomized range finder with power iteration)
- * run on the d x d matrix in shared memory when its result can be certified, else
- * from a parallel Jacobi eigensolver on the whole matrix (SOLAR_ROUTE_AUTO below);
- * s_i = sqrt(lambda_i).  M is accepted for a uniform signature and ignored.
+ * eigenpairs come from a tridiagonal reduction of the d x d matrix (Householder,
+ * Sturm-count multisection, twisted factorisation) when that result can be certified
+ * against G_b, else from a parallel Jacobi eigensolver on the whole matrix
+ * (SOLAR_ROUTE_AUTO above); s_i = sqrt(lambda_i).  Algorithm 1 of the paper (the
+ * randomized range finder) is available as SOLAR_ROUTE_SUBSPACE of
+ * solar_eig_from_partials_ex.  M is accepted for a uniform signature and ignored.
  */
 solar_status_t solar_lowrank_factor(int B, int M, int N, int d, int r, solar_dtype_t dt,
                                     const void* H, float* S, float* V, void* US, int* info,
@@ -143,16 +158,19 @@ int solar_gram_splits(int B, int N, int d, solar_dtype_t dt);
 solar_status_t solar_gram_partials(int B, int N, int d, solar_dtype_t dt, const void* H,
                                    void* workspace, size_t workspace_bytes, void* stream);
 
-/* Sums the partial Grams in slice order and diagonalises; writes S, V, info. */
+/* Sums the partial Grams in slice order and diagonalises; writes S, V, info.  The summed
+ * matrices [B,d,d] fp32 are left in the workspace behind the status words. */
 solar_status_t solar_eig_from_partials(int B, int N, int d, int r, solar_dtype_t dt,
                                        float* S, float* V, int* info,
                                        void* workspace, size_t workspace_bytes, void* stream);
 
 /* As above with the route chosen by the caller.  route_taken (device, [B] ints, or
- * NULL) receives per user: route used (1 subspace, 2 full; 0 = non-finite input)
- * | power steps << 8 | Jacobi sweeps << 16 | reason << 24, where reason says why the
- * range finder was not certified: 1 no gap at the cut, 2 residual too large for its
- * gap, 4 a kept eigenvalue not positive, 8 sweep cap, 16 non-finite pivot. */
+ * NULL) receives per user: route used (1 subspace, 2 full, 3 tridiagonal; 0 = non-finite
+ * input) | power steps << 8 | Jacobi sweeps (route 3: orthogonalisation passes) << 16 |
+ * reason << 24, where reason says why the first route tried was not certified: 1 no gap
+ * at the cut, 2 residual too large for its gap, 4 a kept eigenvalue not positive, 8 sweep
+ * cap, 16 non-finite pivot, 32 vectors of a cluster not independent, 64 trace mismatch
+ * or a non-finite value. */
 solar_status_t solar_eig_from_partials_ex(int B, int N, int d, int r, solar_dtype_t dt, int route,
                                           float* S, float* V, int* info, int* route_taken,
                                           void* workspace, size_t workspace_bytes, void* stream);

@@ -25,17 +25,12 @@
 // rotations it needs from the diagonal blocks of the current matrix, and the matrix is
 // double-buffered, so a round costs ONE barrier.  The 2x2 blocks are stored in four
 // planes so that every access of a warp is free of bank conflicts.
-#include <math.h>
-
-#include "solar_internal.cuh"
+#include "eig_jacobi.cuh"
 
 namespace solar {
 
 namespace {
 
-constexpr float kTolRel = 2.3841858e-07f;  // 2^-22: |g_pq| <= tol*sqrt(g_pp g_qq) counts as zero
-constexpr float kTolAbs = 7.4505806e-09f;  // 2^-27 of the largest diagonal entry
-constexpr float kUnit = 5.9604645e-08f;    // 2^-24, fp32 unit roundoff
 constexpr int kMaxSubspaceIters = 5;       // power steps before the subspace route gives up
 
 // Acceptance thresholds of the subspace route (chosen by the storage type).
@@ -71,57 +66,6 @@ template <int D> struct EigCfg {
   static_assert(DPM_FLOATS <= 2 * D * LD && DPM_FLOATS % 4 == 0, "Zb, Yb, Xb must fit in Gn+Vm");
   static_assert((D * LD) % 4 == 0 && FULL_FLOATS % 4 == 0, "16-byte alignment of the regions");
 };
-
-// Rotation J = [[c, s], [-s, c]] that annihilates g_pq of the 2x2 symmetric block
-// [[a, g], [g, b]]; identity when g is negligible (or not a number).  Returned
-// as s, tau = s/(1+c) and t = s/c: columns are updated in the cancellation-free
-// form x_p' = x_p - s (x_q + tau x_p), x_q' = x_q + s (x_p - tau x_q), and the
-// diagonal as a' = a - t g, b' = b + t g, so a near-identity rotation perturbs
-// the matrix by O(s) instead of by a rounding error of the full entry.
-// `big` is set when the rotated pair had g^2 > stop2 |a b|.  The matrix is scaled so
-// that its largest diagonal entry lies in [1, 2): squares cannot overflow, and entries
-// whose squares underflow are below the absolute threshold.  The approximate rsqrt
-// (2 ulp) only moves the rotation angle by a rounding error.
-struct Rot { float s, tau, t; };
-
-__device__ __forceinline__ Rot jacobi_rot(float a, float b, float g, float thr_abs2, float stop2,
-                                          bool& big) {
-  const float g2 = g * g;
-  const float ab = fabsf(a * b);
-  const bool act = (g2 > thr_abs2) && (g2 > (kTolRel * kTolRel) * ab);
-  big = act && (g2 > stop2 * ab);
-  // With d = b - a and h = sqrt(d^2 + 4 g^2):  cos^2 = (h + |d|) / (2 h),
-  // sin = sgn(d) g / (h cos),  tan = sin / cos,  tau = sin / (1 + cos).
-  // Two dependent special-function evaluations (both rsqrt); 1 / (1 + cos), with
-  // 1 + cos in [1.707, 2], comes from a linear guess and two Newton steps.
-  const float dlt = b - a;
-  const float rh = rsqrtf(fmaf(dlt, dlt, 4.f * g2));
-  const float c2 = fmaf(0.5f * fabsf(dlt), rh, 0.5f);
-  const float rc = rsqrtf(c2);
-  const float c = c2 * rc;
-  const float s = copysignf(g * rh, dlt * g) * rc;
-  const float t = s * rc;
-  const float u = 1.f + c;
-  float y = fmaf(-0.29289f, u, 1.08579f);
-  y = y * fmaf(-u, y, 2.f);
-  y = y * fmaf(-u, y, 2.f);
-  Rot r;
-  r.s = act ? s : 0.f;
-  r.t = act ? t : 0.f;
-  r.tau = act ? s * y : 0.f;
-  return r;
-}
-
-__device__ __forceinline__ void rot_apply(const Rot& r, float& xp, float& xq) {
-  const float p = xp, q = xq;
-  xp = fmaf(-r.s, fmaf(r.tau, p, q), p);
-  xq = fmaf(r.s, fmaf(-r.tau, q, p), q);
-}
-
-// Barrier among the first `nthreads` threads of the CTA (a multiple of 32).
-__device__ __forceinline__ void bar_named(int id, int nthreads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
-}
 
 // Integer mixer (two multiply-xorshift rounds) used as a counter-based generator.
 __device__ __forceinline__ uint32_t mix32(uint32_t x) {
@@ -315,28 +259,7 @@ __device__ __forceinline__ void rows_dot_col(const float* __restrict__ X, const 
 }
 
 // ---- Jacobi on the p x p Rayleigh-Ritz matrix ------------------------------------------
-// Systolic form of the round-robin tournament: the matrix is indexed by SLOT, the pairs of
-// every round are the slots (2i, 2i+1), and after each round a fixed permutation moves the
-// slots (rows and columns of T, columns of W) so that in p-1 rounds every two indices meet
-// once.  Slot 0 stays; slot 1 -> 2; slot 2i -> 2i+2 (1 <= i <= p/2-2); slot p-2 -> p-1;
-// slot 2i+1 -> 2i-1 (i >= 1).  Nothing has to track which original index sits in a slot:
-// eigenvalue and eigenvector simply travel together.
-__device__ __forceinline__ int slot_next(int u, int p) {
-  if (u == 0) return 0;
-  if (u == 1) return 2;
-  if (u & 1) return u - 2;
-  return (u == p - 2) ? p - 1 : u + 2;
-}
-// Offset (in floats) of element (u, v) in the planar 2x2-block layout: block (u/2, v/2), whose
-// four entries sit in four planes [2*(u%2) + v%2][u/2][v/2] with row pitch p/2 + 1, so that
-// every scalar access of a warp (consecutive block columns, or the diagonal) is free of bank
-// conflicts -- both the reads of a thread's own block and the scattered writes of the moved one.
-__device__ __forceinline__ int blk_off(int u, int v, int hp) {
-  return (((u & 1) << 1) + (v & 1)) * (hp * (hp + 1)) + (u >> 1) * (hp + 1) + (v >> 1);
-}
-// Floats of one matrix in that layout.
-__device__ __forceinline__ int blk_size(int hp) { return 4 * hp * (hp + 1); }
-
+// Same systolic tournament as the full route (slot_next), on the small matrix.
 // Layout of the Ritz Jacobi (thread (I, J) = tid / hp, tid % hp: a warp holds 32 / hp whole
 // rows of blocks): row pitch hp and a plane stride of hp * hp plus a small offset.  An
 // exhaustive count over all 18 shared-memory accesses of a round (own block, the two diagonal
@@ -408,41 +331,16 @@ __device__ __forceinline__ int ritz_jacobi(float* Tb, float* Wb, int p, float th
   return sweeps;
 }
 
-// Ranks of lam[0..n) in descending order (ties: lower index first): order[rank] = index.
-__device__ __forceinline__ void rank_descending(const float* lam, int* order, int n, int tid) {
-  if (tid < n) {
-    const float li = lam[tid];
-    int rank = 0;
-    for (int j = 0; j < n; ++j) {
-      const float lj = lam[j];
-      rank += (lj > li) || (lj == li && j < tid);
-    }
-    order[rank] = tid;
-  }
-}
-
-// route_taken[b] = route | power steps << 8 | Jacobi sweeps << 16 | kWhy* bits << 24
-constexpr int kRouteSubspace = 1, kRouteFull = 2;
-// Why the subspace route's result was not certified (0 = it was, or it was not tried):
-constexpr int kWhyCut = 1;          // the trace bound does not separate theta_r from the rest
-constexpr int kWhyResidual = 2;     // a residual is too large for its gap
-constexpr int kWhyNotPositive = 4;  // a kept Ritz value is not positive (rank(H) < r)
-constexpr int kWhySweepCap = 8;     // the Ritz Jacobi hit its sweep cap
-constexpr int kWhyCholesky = 16;    // non-finite pivot in the Cholesky-QR
-
 template <int D>
 __global__ void __launch_bounds__(EigCfg<D>::THREADS, 1)
 eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status, int splits, int r,
-           int p, int route, EigTol tol, float* __restrict__ S, float* __restrict__ V,
-           int* __restrict__ info, int* __restrict__ route_taken) {
+           int p, int route, int sweep_cap, int force_iters, EigTol tol, float* __restrict__ S,
+           float* __restrict__ V, int* __restrict__ info, int* __restrict__ route_taken) {
   using Cfg = EigCfg<D>;
   constexpr int LD = Cfg::LD, NT = Cfg::THREADS;
   extern __shared__ __align__(16) float smem[];
   float* Gc = smem;                 // current matrix
   float* Gn = smem + D * LD;        // next matrix
-  float* Vm = smem + 2 * D * LD;    // accumulated rotations (eigenvectors in columns)
-  float* lam = smem + 3 * D * LD;   // [D] eigenvalues
-  int* order = reinterpret_cast<int*>(lam + D);   // [D] column holding the k-th largest eigenvalue
   __shared__ float s_gmax;
   __shared__ double s_trace;
   __shared__ int s_flags[4];
@@ -559,7 +457,10 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
       __syncthreads();
     }
     const float settle = tol.floor_rel;
-    for (int it = iters; it < kMaxSubspaceIters && ok; ++it) {
+    // force_iters > 0: exactly that many orthonormalised power steps (Algorithm 1 with
+    // n_iter = force_iters - 1), no stopping rule and no retry
+    const int max_it = force_iters > 0 ? min(force_iters, kMaxSubspaceIters) : kMaxSubspaceIters;
+    for (int it = iters; it < max_it && ok; ++it) {
       // Cholesky-QR of the power step's Y = G Z:  A = Y^T Y = L L^T,  Z = Y L^-T
       mul_XtY<D, double, double>(Yb, Yb, Ad, p, LPD, tid, NT);
       __syncthreads();
@@ -577,7 +478,7 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
       mul_XtY<D, float, float>(Zb, Yb, Tc, p, LP, tid, NT);
       __syncthreads();
       iters = it + 1;
-      if (it + 1 == kMaxSubspaceIters) break;
+      if (it + 1 == max_it) break;
       // ||G Z - Z T||_F^2, accumulated per warp then by shared-memory atomics
       if (tid == 0) res2[0] = 0.f;
       __syncthreads();
@@ -601,7 +502,7 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
       const bool settled = sqrtf(res2[0]) <= settle * tmax;
       __syncthreads();
       // with oversampling (p > r) the extra directions never settle: two steps are the rule
-      if (settled || (p > r && it >= 1)) break;
+      if (force_iters == 0 && (settled || (p > r && it >= 1))) break;
     }
 
     if (ok) {
@@ -678,7 +579,7 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
       have_vectors = true;
     }
     // retry only when a residual alone stood in the way and a power step is left
-    if (ok || !have_vectors || s_why != kWhyResidual || iters >= kMaxSubspaceIters) break;
+    if (ok || !have_vectors || s_why != kWhyResidual || iters >= kMaxSubspaceIters || force_iters > 0) break;
     __syncthreads();
     }   // attempts
 
@@ -712,140 +613,12 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
   }
 
   // ============================ route (2): full d x d Jacobi ============================
-  // The same systolic slot form as the Ritz Jacobi, on the whole matrix.  T is kept in the
-  // planar block layout, double-buffered (buffer 0 overlays the row-major G, buffer 1 the
-  // next matrix slot); the eigenvector matrix W stays COLUMN-major and in place: slot v's
-  // vector is column perm[v], the slot move only permutes `perm`.  Lanes run along the row
-  // blocks I, so a warp reads one W column pair as 32 consecutive 8-byte pieces, the column
-  // rotation (and its perm lookup) is uniform across the warp, and every T access is
-  // conflict-free.  Thread (I, Jb) owns the blocks (I, Jb + c*NJ), c < PTJ.
-  {
-    // For d = 64 the four planes lie one word further apart than HP * (HP + 1): counted over every
-    // access of a round that leaves 9 % extra wavefronts from bank conflicts instead of 54 %
-    // (426 -> 384 us for a batch of 64 full solves); for d = 128 the same offset measured slower.
-    constexpr int HP = D / 2, NJ = NT / HP, PTJ = HP / NJ, XP = (HP == 32) ? 1 : 0;
-    constexpr int PLN = HP * (HP + 1) + XP, TBS = 4 * PLN;
-    static_assert(NT % HP == 0 && HP % NJ == 0 && TBS <= D * LD && D * D <= D * LD, "full-route tiling");
-    float* Wc = Vm;                                  // [D cols][D rows]
-    int* perm = order + D;                           // [2][D]
-    const int I = tid % HP, Jb = tid / HP;
-    static_assert(HP == 16 || HP == 32 || HP == 64, "rotation sharing by shuffle");
-
-    float xin[PTJ][4];
-#pragma unroll
-    for (int c = 0; c < PTJ; ++c) {
-      const int J = Jb + c * NJ;
-      xin[c][0] = Gc[(2 * I) * LD + 2 * J];     xin[c][1] = Gc[(2 * I) * LD + 2 * J + 1];
-      xin[c][2] = Gc[(2 * I + 1) * LD + 2 * J]; xin[c][3] = Gc[(2 * I + 1) * LD + 2 * J + 1];
-    }
-    __syncthreads();                                 // all of row-major G is in registers
-    int tdst[PTJ][4];
-    const int r0 = slot_next(2 * I, D), r1 = slot_next(2 * I + 1, D);
-#pragma unroll
-    for (int c = 0; c < PTJ; ++c) {
-      const int J = Jb + c * NJ, src = I * (HP + 1) + J;
-#pragma unroll
-      for (int q = 0; q < 4; ++q) Gc[q * PLN + src] = xin[c][q];
-      const int c0 = slot_next(2 * J, D), c1 = slot_next(2 * J + 1, D);
-      tdst[c][0] = blk_off(r0, c0, HP) + XP * (((r0 & 1) << 1) + (c0 & 1));
-      tdst[c][1] = blk_off(r0, c1, HP) + XP * (((r0 & 1) << 1) + (c1 & 1));
-      tdst[c][2] = blk_off(r1, c0, HP) + XP * (((r1 & 1) << 1) + (c0 & 1));
-      tdst[c][3] = blk_off(r1, c1, HP) + XP * (((r1 & 1) << 1) + (c1 & 1));
-    }
-    for (int e = tid; e < D * D; e += NT) Wc[e] = (e / D == e % D) ? 1.f : 0.f;
-    if (tid < D) perm[tid] = tid;
-    if (tid < 3) s_flags[tid] = 0;
-    __syncthreads();
-
-    const int srcI = I * (HP + 1) + I;
-    int converged = 0, sweeps_done = kMaxSweeps, cur = 0;
-    for (int sweep = 0; sweep < kMaxSweeps; ++sweep) {
-      if (tid == 0) s_flags[(sweep + 1) % 3] = 0;
-      bool worst = false;
-      for (int k = 0; k < D - 1; ++k) {
-        const float* Tc = cur ? Gn : Gc;
-        float* Tn = cur ? Gc : Gn;
-        const int* pc = perm + cur * D;
-        // The lanes of every warp compute the round's HP rotations between them (lane l takes
-        // the pairs l, l + 32, ...); a thread's row rotation is among its own, and the column
-        // rotations, uniform across the warp, come by shuffle -- instead of every thread
-        // computing one rotation per block it owns.
-        constexpr int NR = (HP + 31) / 32;
-        Rot rl[NR];
-#pragma unroll
-        for (int q = 0; q < NR; ++q) {
-          const int pr = (HP >= 32) ? q * 32 + lane : lane % HP;
-          const int sp = pr * (HP + 1) + pr;
-          bool big;
-          rl[q] = jacobi_rot(Tc[sp], Tc[3 * PLN + sp], Tc[PLN + sp], thr_abs2, stop2, big);
-          worst |= big;
-        }
-        Rot rr = rl[0];
-        if (NR == 2 && I >= 32) rr = rl[NR - 1];
-#pragma unroll
-        for (int c = 0; c < PTJ; ++c) {
-          const int J = Jb + c * NJ, src = I * (HP + 1) + J;
-          const Rot& rs = (NR == 2 && J >= 32) ? rl[NR - 1] : rl[0];   // J is uniform across the warp
-          Rot rc;
-          rc.s = __shfl_sync(0xffffffffu, rs.s, J & 31);
-          rc.tau = __shfl_sync(0xffffffffu, rs.tau, J & 31);
-          rc.t = rr.t;                       // used only where I == J
-          float x00 = Tc[src], x01 = Tc[PLN + src], x10 = Tc[2 * PLN + src], x11 = Tc[3 * PLN + src];
-          float2* wa = reinterpret_cast<float2*>(Wc + pc[2 * J] * D + 2 * I);
-          float2* wb = reinterpret_cast<float2*>(Wc + pc[2 * J + 1] * D + 2 * I);
-          float2 va = *wa, vb = *wb;
-          if (I == J) {                      // the pair's own diagonal block
-            const float tg = rc.t * x01;
-            x00 -= tg; x11 += tg;
-            if (rc.s != 0.f) { x01 = 0.f; x10 = 0.f; }
-          } else {
-            rot_apply(rc, x00, x01); rot_apply(rc, x10, x11);   // columns
-            rot_apply(rr, x00, x10); rot_apply(rr, x01, x11);   // rows
-          }
-          rot_apply(rc, va.x, vb.x); rot_apply(rc, va.y, vb.y);
-          Tn[tdst[c][0]] = x00; Tn[tdst[c][1]] = x01; Tn[tdst[c][2]] = x10; Tn[tdst[c][3]] = x11;
-          *wa = va; *wb = vb;
-        }
-        if (tid < D) perm[(cur ^ 1) * D + slot_next(tid, D)] = pc[tid];
-        if (k == D - 2 && worst) s_flags[sweep % 3] = 1;
-        __syncthreads();
-        cur ^= 1;
-      }
-      if (s_flags[sweep % 3] == 0) { converged = 1; sweeps_done = sweep + 1; break; }
-    }
-
-    // ---- order the eigenvalues, keep r, fix the sign of each vector ----------------
-    const float* Tf = cur ? Gn : Gc;
-    const int* pf = perm + cur * D;
-    if (tid < D) lam[tid] = Tf[(tid & 1) * 3 * PLN + (tid >> 1) * (HP + 1) + (tid >> 1)];
-    __syncthreads();
-    rank_descending(lam, order, D, tid);
-    __syncthreads();
-    float* sgn = cur ? Gc : Gn;   // reuse: [r] signs
-    if (tid < r) {
-      const float* col = Wc + pf[order[tid]] * D;
-      float best = -1.f, lead = 1.f;
-      for (int j = 0; j < D; ++j) {
-        const float v = col[j];
-        if (fabsf(v) > best) { best = fabsf(v); lead = v; }   // strict: lowest index wins a tie
-      }
-      sgn[tid] = lead < 0.f ? -1.f : 1.f;
-      S[(size_t)b * r + tid] = sqrtf(fmaxf(lam[order[tid]], 0.f) / sc);
-    }
-    __syncthreads();
-    for (int e = tid; e < D * r; e += NT) {
-      const int j = e / r, i = e % r;
-      V[(size_t)b * D * r + e] = Wc[pf[order[i]] * D + j] * sgn[i];
-    }
-    if (tid == 0) {
-      if (info) info[b] = converged ? 0 : SOLAR_INFO_NOT_CONVERGED;
-      if (route_taken) route_taken[b] = kRouteFull | (sweeps_done << 16) | (s_why << 24);
-    }
-  }
+  full_jacobi_route<D, NT>(smem, s_flags, b, tid, r, sc, thr_abs2, stop2, s_why, sweep_cap, S, V, info,
+                           route_taken);
 }
 
 template <int D>
-cudaError_t launch_d(int B, int r, int p, int route, EigTol tol, const float* gpart,
+cudaError_t launch_d(int B, int r, int p, int route, int sweep_cap, int force_iters, EigTol tol, const float* gpart,
                      const int* gram_status, int splits, float* S, float* V, int* info,
                      int* route_taken, cudaStream_t st) {
   using Cfg = EigCfg<D>;
@@ -854,7 +627,7 @@ cudaError_t launch_d(int B, int r, int p, int route, EigTol tol, const float* gp
                                        (int)Cfg::SMEM);
   if (e != cudaSuccess) return e;
   return launch_pdl(eig_kernel<D>, dim3(B), dim3(Cfg::THREADS), Cfg::SMEM, st, gpart, gram_status, splits,
-                    r, p, route, tol, S, V, info, route_taken);
+                    r, p, route, sweep_cap, force_iters, tol, S, V, info, route_taken);
 }
 
 }  // namespace
@@ -867,9 +640,14 @@ int eig_subspace_dim(int d, int r) {
   return (p <= 32 && 2 * p <= d) ? p : 0;
 }
 
-cudaError_t launch_eig(int B, int d, int r, solar_dtype_t dt, int route, const float* gpart,
-                       const int* gram_status, int splits, float* S, float* V, int* info,
-                       int* route_taken, cudaStream_t st) {
+cudaError_t launch_eig(int B, int d, int r, solar_dtype_t dt, int route, int sweep_cap, int force_iters,
+                       const float* gpart, const int* gram_status, int splits, float* gsum, float* S,
+                       float* V, int* info, int* route_taken, cudaStream_t st) {
+  if (sweep_cap <= 0 || sweep_cap > kMaxSweeps) sweep_cap = kMaxSweeps;
+  // AUTO and TRIDIAG: the tridiagonal route (with the Jacobi solve behind it in AUTO)
+  if (route == SOLAR_ROUTE_AUTO || route == SOLAR_ROUTE_TRIDIAG)
+    return launch_eig_tridiag(B, d, r, dt, route, sweep_cap, gpart, gram_status, splits, gsum, S, V, info,
+                              route_taken, st);
   EigTol tol;
   if (dt == SOLAR_BF16) {
     tol.eps_vec = 1e-3f; tol.floor_rel = 256.f * kUnit; tol.sweep_stop = 1e-3f;
@@ -878,9 +656,9 @@ cudaError_t launch_eig(int B, int d, int r, solar_dtype_t dt, int route, const f
   }
   const int p = eig_subspace_dim(d, r);
   switch (d) {
-    case 32: return launch_d<32>(B, r, p, route, tol, gpart, gram_status, splits, S, V, info, route_taken, st);
-    case 64: return launch_d<64>(B, r, p, route, tol, gpart, gram_status, splits, S, V, info, route_taken, st);
-    case 128: return launch_d<128>(B, r, p, route, tol, gpart, gram_status, splits, S, V, info, route_taken, st);
+    case 32: return launch_d<32>(B, r, p, route, sweep_cap, force_iters, tol, gpart, gram_status, splits, S, V, info, route_taken, st);
+    case 64: return launch_d<64>(B, r, p, route, sweep_cap, force_iters, tol, gpart, gram_status, splits, S, V, info, route_taken, st);
+    case 128: return launch_d<128>(B, r, p, route, sweep_cap, force_iters, tol, gpart, gram_status, splits, S, V, info, route_taken, st);
     default: return cudaErrorInvalidValue;
   }
 }

@@ -79,8 +79,8 @@ solar_status_t solar_eig_from_partials_ex(int B, int N, int d, int r, solar_dtyp
                                           float* S, float* V, int* info, int* route_taken,
                                           void* workspace, size_t workspace_bytes, void* stream) {
   SOLAR_TRY(check_dims(B, 0, N, d, r, dt));
-  if (route != SOLAR_ROUTE_AUTO && route != SOLAR_ROUTE_SUBSPACE && route != SOLAR_ROUTE_FULL)
-    return SOLAR_ERR_INVALID_ARG;
+  const int base_route = route & 0xff, sweep_cap = (route >> 8) & 0xff, force_iters = (route >> 16) & 0xff;
+  if ((route & ~0xffffff) != 0 || base_route > SOLAR_ROUTE_TRIDIAG) return SOLAR_ERR_INVALID_ARG;
   if (B == 0) return SOLAR_OK;
   SOLAR_TRY(check_ptr(S));
   SOLAR_TRY(check_ptr(V));
@@ -91,8 +91,10 @@ solar_status_t solar_eig_from_partials_ex(int B, int N, int d, int r, solar_dtyp
   const GramPlan plan = gram_plan(B, N);
   const int* status =
       reinterpret_cast<const int*>(static_cast<const char*>(workspace) + gram_status_offset(B, N, d));
-  return from_cuda(launch_eig(B, d, r, dt, route, static_cast<const float*>(workspace), status,
-                              plan.splits, S, V, info, route_taken, static_cast<cudaStream_t>(stream)));
+  float* gsum = reinterpret_cast<float*>(static_cast<char*>(workspace) + gram_sum_offset(B, N, d));
+  return from_cuda(launch_eig(B, d, r, dt, base_route, sweep_cap, force_iters, static_cast<const float*>(workspace),
+                              status, plan.splits, gsum, S, V, info, route_taken,
+                              static_cast<cudaStream_t>(stream)));
 }
 
 solar_status_t solar_eig_from_partials(int B, int N, int d, int r, solar_dtype_t dt, float* S,

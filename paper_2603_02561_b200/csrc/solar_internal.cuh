@@ -54,9 +54,14 @@ inline size_t gram_status_offset(int B, int N, int d) {
   const GramPlan p = gram_plan(B, N);
   return align_up((size_t)B * p.splits * d * d * sizeof(float), 256);
 }
-inline size_t factor_ws_bytes(int B, int N, int d) {
+// Behind the status words: the summed Gram matrices [B][d][d] fp32, written by the eigensolver
+// (its residual check and its Jacobi fallback read them back).
+inline size_t gram_sum_offset(int B, int N, int d) {
   const GramPlan p = gram_plan(B, N);
   return gram_status_offset(B, N, d) + align_up((size_t)B * p.splits * sizeof(int), 256);
+}
+inline size_t factor_ws_bytes(int B, int N, int d) {
+  return gram_sum_offset(B, N, d) + align_up((size_t)B * d * d * sizeof(float), 256);
 }
 
 // Workspace of the attention call, per user (all segments 256-byte aligned):
@@ -141,9 +146,12 @@ cudaError_t launch_gram_simt(int B, int N, int d, solar_dtype_t dt, const void* 
 bool gram_umma_supported(int N, int d, solar_dtype_t dt);
 cudaError_t launch_gram_umma(int B, int N, int d, const void* H, float* gpart, int* status,
                              const GramPlan& plan, cudaStream_t st);
-cudaError_t launch_eig(int B, int d, int r, solar_dtype_t dt, int route, const float* gpart,
-                       const int* gram_status, int splits, float* S, float* V, int* info,
-                       int* route_taken, cudaStream_t st);
+cudaError_t launch_eig(int B, int d, int r, solar_dtype_t dt, int route, int sweep_cap, int force_iters,
+                       const float* gpart, const int* gram_status, int splits, float* gsum, float* S,
+                       float* V, int* info, int* route_taken, cudaStream_t st);
+cudaError_t launch_eig_tridiag(int B, int d, int r, solar_dtype_t dt, int route, int sweep_cap,
+                               const float* gpart, const int* gram_status, int splits, float* gsum,
+                               float* S, float* V, int* info, int* route_taken, cudaStream_t st);
 int eig_subspace_dim(int d, int r);
 cudaError_t launch_project_us(int B, int N, int d, int r, solar_dtype_t dt, const void* H,
                               const float* V, void* US, cudaStream_t st);

@@ -18,7 +18,12 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA = range(5)
 F32, BF16 = 0, 1
 FLAG_NO_SOFTMAX = 1
 INFO_NOT_CONVERGED, INFO_NONFINITE, INFO_NOT_CERTIFIED, INFO_DEVICE_WAIT = 1, 2, 4, 8
-ROUTE_AUTO, ROUTE_SUBSPACE, ROUTE_FULL = 0, 1, 2
+ROUTE_AUTO, ROUTE_SUBSPACE, ROUTE_FULL, ROUTE_TRIDIAG = 0, 1, 2, 3
+
+
+def route_with(route: int, sweep_cap: int = 0, power_steps: int = 0) -> int:
+    """The route argument of eig_from_partials_ex with its optional fields (SOLAR_ROUTE_WITH)."""
+    return int(route) | (int(sweep_cap) << 8) | (int(power_steps) << 16)
 
 _c_int, _c_size, _c_vp, _c_float, _c_uint = (ctypes.c_int, ctypes.c_size_t, ctypes.c_void_p,
                                               ctypes.c_float, ctypes.c_uint)
