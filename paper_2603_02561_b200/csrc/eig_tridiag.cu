@@ -1,23 +1,27 @@
 // Batched symmetric eigensolver, tridiagonal route: the top-r eigenpairs of every Gram matrix
 // G_b = H_b^T H_b (Eq. 9 without U: s_i = sqrt(lambda_i), V = eigenvectors) by the classical
-// dense-symmetric chain, one CTA per user, sized so that a user costs a few tens of thousands
-// of warp instructions instead of a few hundred thousand for a Jacobi solve:
+// dense-symmetric chain, one CTA per user, sized so that a user costs tens of thousands of warp
+// instructions and a modest register and shared-memory footprint (several CTAs share an SM with
+// the streaming kernels of other requests) instead of the hundreds of thousands of a Jacobi solve:
 //
 //   1. G = sum of the slices' partial Grams (fixed order), scaled by a power of two.
-//   2. Householder tridiagonalisation T = Q^T G Q with the matrix held in REGISTERS: one row
-//      (d = 32, 128) or two rows (d = 64) per lane of the warps that take part, so the
-//      symmetric matrix-vector product and the rank-2 update of a step are lane-local FMAs on
-//      statically indexed registers; a step needs two reductions (the column norm and p^T v)
-//      and, with one warp, no CTA barrier at all.
-//   3. The r largest eigenvalues of T by multisection on Sturm counts (one lane per
-//      eigenvalue, three interior points per step: two bits per step), the counts taken from
-//      the three-term recurrence of the leading principal minors with a power-of-two rescale
-//      every four steps -- one FMA per step on the dependency chain instead of a division.
-//   4. One eigenvector per lane from the twisted factorisation of T - lambda I (forward and
-//      backward pivot sequences, twist at the smallest |gamma_k|): inverse iteration from the
-//      best unit vector, O(d) per vector, no pivoting.
-//   5. Back-transformation V = Q Z, each lane applying the d-2 reflectors to its own vector
-//      held in registers.
+//   2. Householder tridiagonalisation T = Q^T G Q with the matrix held in REGISTERS, spread over
+//      all warps of the CTA: thread (warp w, lane l) owns rows l, l+32, ... and the columns of
+//      its warp's 4-column groups, so the symmetric matrix-vector product and the rank-2 update
+//      of a step are FMAs on statically indexed registers.  Every warp computes the step's
+//      scalars redundantly (column norm and p^T v by shuffles); the warps exchange only their
+//      partial products, through shared memory, at ONE barrier per step.  The next step's
+//      column comes from the owner of row k+1 (by symmetry) before the update and is corrected
+//      by the rank-2 term, so no step waits for the update of the one before.
+//   3. The r largest eigenvalues of T by multisection on Sturm counts: one lane per eigenvalue,
+//      one interior point per warp and step (4 or 8 points), the counts taken from the
+//      three-term recurrence of the leading principal minors with a power-of-two rescale every
+//      four steps -- one FMA per step on the dependency chain instead of a division.
+//   4. One eigenvector per eigenvalue from the twisted factorisation of T - lambda I (forward
+//      and backward pivot sequences as ratios of consecutive minors, twist at the smallest
+//      |gamma_k|): inverse iteration from the best unit vector, O(d) per vector, no pivoting.
+//   5. Back-transformation V = Q Z: four threads per vector, each applying the d-2 reflectors to
+//      its quarter of the rows held in registers.
 //   6. A first-order symmetric orthogonalisation V <- V (I - (V^T V - I)/2), repeated while
 //      V^T V - I is above the rounding level (vectors of close eigenvalues come out of step 4
 //      with a mutual error of order eps |T| / gap).
@@ -26,6 +30,11 @@
 //      at the rounding floor), V^T V = I to rounding, and trace(T) = trace(G); otherwise the
 //      CTA runs the parallel Jacobi eigensolver on the whole matrix, which is valid for any
 //      spectrum (clusters of equal eigenvalues, rank(H) < r, ...).
+//
+// A warp that runs alone on its scheduler pays the full latency of every branch and of every
+// dependent instruction; the code below is therefore straight-line over static ranges (the
+// Householder loop is cut into stages with fixed live rows and columns), keeps divisions off
+// the dependency chains, and spreads independent work over the warps.
 #include "eig_jacobi.cuh"
 
 namespace solar {
@@ -37,36 +46,41 @@ constexpr unsigned kFull = 0xffffffffu;
 template <int D> struct TriCfg {
   static constexpr int NT = (D == 128) ? 256 : 128;   // threads of the CTA
   static constexpr int NW = NT / 32;
-  static constexpr int TW = (D == 128) ? 4 : 1;       // warps that hold the matrix while it is reduced
-  static constexpr int RPL = (D == 64) ? 2 : 1;       // rows per lane
+  static constexpr int RPT = D / 32;                  // rows per thread: l + 32 q
+  static constexpr int CPT = D / NW;                  // columns per thread ...
+  static constexpr int NG = CPT / 4;                  // ... as 4-column groups: group g of warp w = columns 4 (w + NW g) ..+3
+  static constexpr int SS = 4 * NW;                   // steps per stage: from step s * SS on, the groups g < s are finished
   static constexpr int LD = D + 4;                    // pitch of the staged row-major G
   static constexpr int NB = D / 4;                    // 4-column blocks of a row
-  static_assert(TW * 32 * RPL == D, "every row has an owner");
+  static_assert(SS * NG == D && RPT * 32 == D, "ownership covers the matrix");
 };
 
 // Shared-memory layout (floats) for subspace width RP = 32 * ceil(r / 32).
 template <int D, int RP> struct TriSmem {
   using C = TriCfg<D>;
   static constexpr int HV = 0;                                   // [D][D] reflector k in row k; later G
-  static constexpr int VS = HV + D * D;                          // [D][RP] tridiagonal vectors, then V
+  static constexpr int VS = HV + D * D;                          // [D][RP] V
   static constexpr int WORK_FLOATS = (D * C::LD > 2 * D * RP) ? D * C::LD : 2 * D * RP;
   static constexpr int WORK = VS + D * RP;                       // staged G | tf, tb [D][RP] | V'
-  static constexpr int EM = WORK + WORK_FLOATS;                  // [RP][RP] V^T V - I
+  static constexpr int EM = WORK + WORK_FLOATS;                  // [RP][RP] V^T V - I (before: multisection flags)
   static constexpr int DG = EM + RP * RP;                        // [D] diagonal of T
   static constexpr int EO = DG + D;                              // [D] off-diagonal: e[k] couples k, k+1
   static constexpr int E2 = EO + D;                              // [D] e2s[i] = e[i-1]^2 (floored), e2s[0] = 0
   static constexpr int BE = E2 + D;                              // [D] beta of reflector k
-  static constexpr int WV = BE + D;                              // [D] w of the current step
-  static constexpr int LAM = WV + D;                             // [RP] eigenvalues of T
+  static constexpr int XP = BE + D;                              // [2][D] row k+1 before the update of step k
+  static constexpr int TP = XP + 2 * D;                          // [2][NW][D] the warps' partial products A v
+  static constexpr int PV = TP + 2 * C::NW * D;                  // [2][8] the warps' partial p^T v
+  static constexpr int LAM = PV + 16;                            // [RP] eigenvalues of T
   static constexpr int TH = LAM + RP;                            // [RP] Rayleigh quotients
   static constexpr int RH = TH + RP;                             // [RP] squared residual norms
-  static constexpr int SG = RH + RP;                             // [RP] gauge signs
-  static constexpr int PART = SG + RP;                           // [NW][RP] per-warp partial sums
-  static constexpr int TRI_FLOATS = PART + C::NW * RP;
+  static constexpr int SG = RH + RP;                             // [RP] gauge signs; before: 1 / |z|
+  static constexpr int KT = SG + RP;                             // [RP] twist index (int)
+  static constexpr int PART = KT + RP;                           // [2][NW][RP] per-warp partial results
+  static constexpr int TRI_FLOATS = PART + 2 * C::NW * RP;
   static constexpr int FLOATS = TRI_FLOATS > full_jacobi_floats<D>() ? TRI_FLOATS : full_jacobi_floats<D>();
   static constexpr size_t BYTES = (size_t)FLOATS * sizeof(float);
-  static_assert(DG % 4 == 0 && EO % 4 == 0 && E2 % 4 == 0 && WV % 4 == 0 && EM % 4 == 0 && WORK % 4 == 0 &&
-                VS % 4 == 0, "16-byte alignment of the regions");
+  static_assert(DG % 4 == 0 && EO % 4 == 0 && E2 % 4 == 0 && XP % 4 == 0 && TP % 4 == 0 && PV % 4 == 0 &&
+                EM % 4 == 0 && WORK % 4 == 0 && VS % 4 == 0, "16-byte alignment of the regions");
 };
 
 __device__ __forceinline__ float warp_sum(float v) {
@@ -79,11 +93,182 @@ __device__ __forceinline__ float warp_max(float v) {
   for (int o = 16; o; o >>= 1) v = fmaxf(v, __shfl_xor_sync(kFull, v, o));
   return v;
 }
-__device__ __forceinline__ float pick4(const float4& v, int c) {
-  return c == 0 ? v.x : c == 1 ? v.y : c == 2 ? v.z : v.w;
+// 16-byte store to shared memory under a predicate, without a branch.
+__device__ __forceinline__ void sts_v4_if(float* p, float a, float b, float c, float d, bool pred) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.s32 p, %5, 0;\n\t@p st.shared.v4.f32 [%0], {%1, %2, %3, %4};\n\t}"
+               ::"r"((uint32_t)__cvta_generic_to_shared(p)), "f"(a), "f"(b), "f"(c), "f"(d), "r"((int)pred)
+               : "memory");
 }
-__device__ __forceinline__ void put4(float4& v, int c, float x) {
-  if (c == 0) v.x = x; else if (c == 1) v.y = x; else if (c == 2) v.z = x; else v.w = x;
+// 1 / sqrt(x) and 1 / x to fp32 accuracy (approximation plus one Newton step): the reflector
+// I - beta v v^T is orthogonal only as far as beta v^T v = 2 holds.
+__device__ __forceinline__ float rsqrt_acc(float x) {
+  const float y = rsqrtf(x);
+  return y * fmaf(-0.5f * x * y, y, 1.5f);
+}
+__device__ __forceinline__ float rcp_acc(float x) {
+  float y;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y * fmaf(-x, y, 2.f);
+}
+
+// ---- Householder steps of stage S: k in [S * SS, min((S + 1) * SS, D - 2)) -------------------
+// From step S * SS on the column groups g < S and the row slots q < Q0 are finished, so every
+// range below is static.  State carried from step to step: the matrix a, and column k of the
+// current matrix at the thread's rows (xr) and columns (xc; by symmetry row k).
+template <int D, int S>
+__device__ __forceinline__ void tri_stage(float (&a)[TriCfg<D>::RPT][TriCfg<D>::CPT], float (&xr)[TriCfg<D>::RPT],
+                                          float (&xc)[TriCfg<D>::CPT], float* __restrict__ hv,
+                                          float* __restrict__ xpre, float* __restrict__ tpart,
+                                          float* __restrict__ pvp, float* __restrict__ dg, float* __restrict__ eo,
+                                          float* __restrict__ betas, int tid) {
+  using C = TriCfg<D>;
+  constexpr int NW = C::NW, RPT = C::RPT, NG = C::NG, SS = C::SS;
+  constexpr int G0 = S;                                               // first live column group
+  constexpr int Q0 = (S * SS >= 31) ? (S * SS - 31) / 32 + 1 : 0;     // first live row slot
+  constexpr int K1 = ((S + 1) * SS < D - 2) ? (S + 1) * SS : D - 2;
+  const int lane = tid & 31, warp = tid >> 5;
+#pragma unroll 1
+  for (int k = S * SS; k < K1; ++k) {
+    const int k1 = k + 1, par = k & 1, q1 = k1 >> 5, l1 = k1 & 31;
+    // row k+1 of the current matrix at my columns, for the next step's vector (no branch: the
+    // store is predicated; one lane per warp owns the row)
+#pragma unroll
+    for (int q = Q0; q < RPT; ++q)
+#pragma unroll
+      for (int g = G0; g < NG; ++g)
+        sts_v4_if(xpre + par * D + 4 * (warp + NW * g), a[q][4 * g], a[q][4 * g + 1], a[q][4 * g + 2],
+                  a[q][4 * g + 3], q == q1 && lane == l1);
+    // x = column k below the subdiagonal; its norm; alpha, beta, v
+    float xs[RPT], sq = 0.f, c1 = xr[RPT - 1], ck = xr[RPT - 1];
+#pragma unroll
+    for (int q = RPT - 1; q >= 0; --q) {
+      xs[q] = (q >= Q0 && lane + 32 * q > k1) ? xr[q] : 0.f;
+      sq = fmaf(xs[q], xs[q], sq);
+      c1 = (q == q1) ? xr[q] : c1;
+      ck = (q == (k >> 5)) ? xr[q] : ck;
+    }
+    const float x1 = __shfl_sync(kFull, c1, l1), dk = __shfl_sync(kFull, ck, k & 31);
+    const float tail2 = warp_sum(sq);
+    // With nothing to annihilate (an exactly zero tail) the reflector is the identity: beta = 0
+    // makes p, w and the update vanish, and the step still hands on column k+1.
+    const bool reflect = tail2 > 1e-35f;
+    const float s2 = fmaf(x1, x1, tail2);
+    const float nrm = s2 * rsqrt_acc(fmaxf(s2, 1e-37f));
+    const float alpha = reflect ? -copysignf(nrm, x1) : x1;
+    const float vk1 = reflect ? x1 - alpha : 0.f;
+    const float beta = reflect ? rcp_acc(nrm * fabsf(vk1)) : 0.f;
+    if (tid == 0) { dg[k] = dk; eo[k] = alpha; betas[k] = beta; }
+    float vr[RPT], vc[NG][4];
+#pragma unroll
+    for (int q = Q0; q < RPT; ++q) {
+      vr[q] = (lane + 32 * q == k1) ? vk1 : xs[q];
+      if (warp == 0) hv[k * D + lane + 32 * q] = vr[q];        // reflector k (rows <= k stay zero)
+    }
+#pragma unroll
+    for (int g = G0; g < NG; ++g)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const int col = 4 * (warp + NW * g) + c;
+        vc[g][c] = (col == k1) ? vk1 : (col > k1 ? xc[4 * g + c] : 0.f);
+      }
+    // my columns' share of A v at my rows, and of p^T v
+    float dp = 0.f;
+#pragma unroll
+    for (int q = Q0; q < RPT; ++q) {
+      float t0 = 0.f, t1 = 0.f;
+#pragma unroll
+      for (int g = G0; g < NG; ++g) {
+        t0 = fmaf(a[q][4 * g], vc[g][0], t0);     t1 = fmaf(a[q][4 * g + 1], vc[g][1], t1);
+        t0 = fmaf(a[q][4 * g + 2], vc[g][2], t0); t1 = fmaf(a[q][4 * g + 3], vc[g][3], t1);
+      }
+      const float pq = t0 + t1;
+      tpart[(par * NW + warp) * D + lane + 32 * q] = pq;
+      dp = fmaf(pq, vr[q], dp);
+    }
+    dp = warp_sum(dp);
+    if (lane == 0) pvp[par * 8 + warp] = dp;
+    __syncthreads();
+    // p = beta A v at my rows, my columns and at k+1; K = beta p^T v / 2; w = p - K v
+    float pvs = 0.f, pk1 = 0.f;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) { pvs += pvp[par * 8 + w]; pk1 += tpart[(par * NW + w) * D + k1]; }
+    const float kk = 0.5f * beta * beta * pvs;
+    const float wk1 = fmaf(-kk, vk1, beta * pk1);
+    float wr[RPT], wc[NG][4];
+#pragma unroll
+    for (int q = Q0; q < RPT; ++q) {
+      float t = 0.f;
+#pragma unroll
+      for (int w = 0; w < NW; ++w) t += tpart[(par * NW + w) * D + lane + 32 * q];
+      wr[q] = (lane + 32 * q > k) ? fmaf(-kk, vr[q], beta * t) : 0.f;
+      // column k+1 of the updated matrix at my rows: row k+1 before the update, corrected
+      xr[q] = fmaf(-wr[q], vk1, fmaf(-vr[q], wk1, xpre[par * D + lane + 32 * q]));
+    }
+#pragma unroll
+    for (int g = G0; g < NG; ++g) {
+      const int cb = 4 * (warp + NW * g);
+      float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int w = 0; w < NW; ++w) {
+        const float4 u = *reinterpret_cast<const float4*>(tpart + (par * NW + w) * D + cb);
+        t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
+      }
+      const float4 xp = *reinterpret_cast<const float4*>(xpre + par * D + cb);
+      const float tt[4] = {t.x, t.y, t.z, t.w}, xx[4] = {xp.x, xp.y, xp.z, xp.w};
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        wc[g][c] = (cb + c > k) ? fmaf(-kk, vc[g][c], beta * tt[c]) : 0.f;
+        xc[4 * g + c] = fmaf(-wc[g][c], vk1, fmaf(-vc[g][c], wk1, xx[c]));
+      }
+    }
+    // A <- A - v w^T - w v^T on the live block
+#pragma unroll
+    for (int q = Q0; q < RPT; ++q)
+#pragma unroll
+      for (int g = G0; g < NG; ++g)
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          a[q][4 * g + c] = fmaf(-vr[q], wc[g][c], fmaf(-wr[q], vc[g][c], a[q][4 * g + c]));
+  }
+}
+
+// Number of eigenvalues of T below x, for CH values of x at once.  p_{i+1} = (d_i - x) p_i -
+// e_{i-1}^2 p_{i-1} is the leading principal minor of order i+1 of T - x I; the sign changes
+// along p_0 = 1, p_1, ..., p_D count the eigenvalues below x.  The off-diagonal squares are
+// floored above zero, so an exact zero never persists, and an isolated zero gives one change
+// whichever sign the hardware gives it.
+template <int D, int CH>
+__device__ __forceinline__ void sturm(const float* __restrict__ dg, const float* __restrict__ e2s,
+                                      const float (&x)[CH], int (&cnt)[CH]) {
+  float p[CH], q[CH];
+  unsigned n[CH];
+#pragma unroll
+  for (int h = 0; h < CH; ++h) { p[h] = 1.f; q[h] = 0.f; n[h] = 0; }
+#pragma unroll 4
+  for (int ib = 0; ib < D / 4; ++ib) {
+    const float4 d4 = *reinterpret_cast<const float4*>(dg + 4 * ib);
+    const float4 e4 = *reinterpret_cast<const float4*>(e2s + 4 * ib);
+    const float dd[4] = {d4.x, d4.y, d4.z, d4.w}, ee[4] = {e4.x, e4.y, e4.z, e4.w};
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+      for (int h = 0; h < CH; ++h) {
+        const float t = ee[u] * q[h];
+        const float rr = fmaf(dd[u] - x[h], p[h], -t);
+        n[h] += (__float_as_uint(rr) ^ __float_as_uint(p[h])) >> 31;
+        q[h] = p[h]; p[h] = rr;
+      }
+    // bring the larger of (p, q) back into [1, 2): |d - x| and e^2 are bounded by the scaling of G,
+    // so four steps can neither overflow nor (factors above 2^-23 each) underflow
+#pragma unroll
+    for (int h = 0; h < CH; ++h) {
+      const unsigned m = __float_as_uint(fmaxf(fabsf(p[h]), fabsf(q[h]))) >> 23;
+      const float sc = __uint_as_float((254u - m) << 23);
+      p[h] *= sc; q[h] *= sc;
+    }
+  }
+#pragma unroll
+  for (int h = 0; h < CH; ++h) cnt[h] = (int)n[h];
 }
 
 // Acceptance thresholds (chosen by the storage type).
@@ -94,44 +279,6 @@ struct TriTol {
   float sweep_stop;  // of the Jacobi fallback
 };
 
-// Number of eigenvalues of T below x, for three values of x at once.  p_{i+1} = (d_i - x) p_i -
-// e_{i-1}^2 p_{i-1} is the leading principal minor of order i+1 of T - x I; the sign changes
-// along p_0 = 1, p_1, ..., p_D count the eigenvalues below x.  The off-diagonal squares are
-// floored above zero, so an exact zero never persists, and an isolated zero gives one change
-// whichever sign the hardware gives it.
-template <int D>
-__device__ __forceinline__ void sturm3(const float* __restrict__ dg, const float* __restrict__ e2s,
-                                       float x0, float x1, float x2, int& c0, int& c1, int& c2) {
-  float p0 = 1.f, p1 = 1.f, p2 = 1.f, q0 = 0.f, q1 = 0.f, q2 = 0.f;
-  unsigned n0 = 0, n1 = 0, n2 = 0;
-#pragma unroll 2
-  for (int ib = 0; ib < D / 4; ++ib) {
-    const float4 d4 = *reinterpret_cast<const float4*>(dg + 4 * ib);
-    const float4 e4 = *reinterpret_cast<const float4*>(e2s + 4 * ib);
-    const float dd[4] = {d4.x, d4.y, d4.z, d4.w}, ee[4] = {e4.x, e4.y, e4.z, e4.w};
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const float t0 = ee[u] * q0, t1 = ee[u] * q1, t2 = ee[u] * q2;
-      const float r0 = fmaf(dd[u] - x0, p0, -t0);
-      const float r1 = fmaf(dd[u] - x1, p1, -t1);
-      const float r2 = fmaf(dd[u] - x2, p2, -t2);
-      n0 += (__float_as_uint(r0) ^ __float_as_uint(p0)) >> 31;
-      n1 += (__float_as_uint(r1) ^ __float_as_uint(p1)) >> 31;
-      n2 += (__float_as_uint(r2) ^ __float_as_uint(p2)) >> 31;
-      q0 = p0; p0 = r0; q1 = p1; p1 = r1; q2 = p2; p2 = r2;
-    }
-    // bring the larger of (p, q) back into [1, 2): |d - x| and e^2 are bounded by the scaling of G,
-    // so four steps can neither overflow nor (factors above 2^-23 each) underflow
-    const unsigned m0 = __float_as_uint(fmaxf(fabsf(p0), fabsf(q0))) >> 23;
-    const unsigned m1 = __float_as_uint(fmaxf(fabsf(p1), fabsf(q1))) >> 23;
-    const unsigned m2 = __float_as_uint(fmaxf(fabsf(p2), fabsf(q2))) >> 23;
-    const float s0 = __uint_as_float((254u - m0) << 23), s1 = __uint_as_float((254u - m1) << 23);
-    const float s2 = __uint_as_float((254u - m2) << 23);
-    p0 *= s0; q0 *= s0; p1 *= s1; q1 *= s1; p2 *= s2; q2 *= s2;
-  }
-  c0 = (int)n0; c1 = (int)n1; c2 = (int)n2;
-}
-
 template <int D, int RP>
 __global__ void __launch_bounds__(TriCfg<D>::NT, 1)
 eig_tridiag_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status, int splits,
@@ -140,8 +287,9 @@ eig_tridiag_kernel(const float* __restrict__ gpart, const int* __restrict__ gram
                    int* __restrict__ route_taken) {
   using Cfg = TriCfg<D>;
   using L = TriSmem<D, RP>;
-  constexpr int NT = Cfg::NT, NW = Cfg::NW, TW = Cfg::TW, RPL = Cfg::RPL, LD = Cfg::LD, NB = Cfg::NB;
-  constexpr int NE = RP / 32;                 // eigenvalues (columns) per lane in the column-parallel phases
+  constexpr int NT = Cfg::NT, NW = Cfg::NW, RPT = Cfg::RPT, CPT = Cfg::CPT, NG = Cfg::NG, LD = Cfg::LD;
+  constexpr int NE = RP / 32;                 // groups of 32 eigenvalues (columns)
+  constexpr int WG = NW / NE;                 // warps per group in the eigenvalue-parallel phases
   extern __shared__ __align__(16) float smem[];
   float* hv = smem + L::HV;
   float* vs = smem + L::VS;
@@ -151,16 +299,17 @@ eig_tridiag_kernel(const float* __restrict__ gpart, const int* __restrict__ gram
   float* eo = smem + L::EO;
   float* e2s = smem + L::E2;
   float* betas = smem + L::BE;
-  float* wv = smem + L::WV;
+  float* xpre = smem + L::XP;
+  float* tpart = smem + L::TP;
+  float* pvp = smem + L::PV;
   float* lamv = smem + L::LAM;
   float* theta = smem + L::TH;
   float* rho2 = smem + L::RH;
   float* sgn = smem + L::SG;
+  int* ktv = reinterpret_cast<int*>(smem + L::KT);
   float* part = smem + L::PART;
   __shared__ float s_gmax, s_lo, s_hi, s_emax, s_trT;
   __shared__ double s_trace;
-  __shared__ float s_red[2][4];
-  __shared__ float s_scal[2];
   __shared__ int s_flags[4];
   __shared__ int s_why;
 
@@ -175,28 +324,39 @@ eig_tridiag_kernel(const float* __restrict__ gpart, const int* __restrict__ gram
     int lost = 0;
     for (int s = tid; s < splits; s += NT) lost |= (gram_status[b * splits + s] != kGramStatusOk);
     int bad = 0;
-    for (int e = tid; e < D * D / 4; e += NT) {
-      // fp32 sums in a fixed order (GW slices at a time, pairwise within the group); all loads of a
-      // group are issued before the first add: the loop is bound by their latency
-      constexpr int GW = 16;
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    // fp32 sums in a fixed order (GW slices at a time, pairwise within the group); all loads of a
+    // group, for two elements, are issued before the first add: the loop is bound by their latency
+    static_assert((D * D / 4) % (2 * NT) == 0, "two elements per thread and trip");
+    for (int e = tid; e < D * D / 4; e += 2 * NT) {
+      constexpr int GW = 8;
+      float4 acc[2] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
       for (int s = 0; s < splits; s += GW) {
-        float4 v[GW];
+        float4 v[2][GW];
 #pragma unroll
-        for (int u = 0; u < GW; ++u)
-          v[u] = (s + u < splits) ? __ldg(gp + (size_t)(s + u) * (D * D / 4) + e)
-                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int h = 0; h < 2; ++h)
 #pragma unroll
-        for (int h = GW / 2; h >= 1; h >>= 1)
+          for (int u = 0; u < GW; ++u)
+            v[h][u] = (s + u < splits) ? __ldg(gp + (size_t)(s + u) * (D * D / 4) + e + h * NT)
+                                       : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-          for (int u = 0; u < h; ++u) {
-            v[u].x += v[u + h].x; v[u].y += v[u + h].y; v[u].z += v[u + h].z; v[u].w += v[u + h].w;
-          }
-        acc.x += v[0].x; acc.y += v[0].y; acc.z += v[0].z; acc.w += v[0].w;
+        for (int h = 0; h < 2; ++h) {
+#pragma unroll
+          for (int w = GW / 2; w >= 1; w >>= 1)
+#pragma unroll
+            for (int u = 0; u < w; ++u) {
+              v[h][u].x += v[h][u + w].x; v[h][u].y += v[h][u + w].y;
+              v[h][u].z += v[h][u + w].z; v[h][u].w += v[h][u + w].w;
+            }
+          acc[h].x += v[h][0].x; acc[h].y += v[h][0].y; acc[h].z += v[h][0].z; acc[h].w += v[h][0].w;
+        }
       }
-      bad |= !(isfinite(acc.x) && isfinite(acc.y) && isfinite(acc.z) && isfinite(acc.w));
-      *reinterpret_cast<float4*>(Gs + (e / (D / 4)) * LD + (e % (D / 4)) * 4) = acc;
-      reinterpret_cast<float4*>(gout)[e] = acc;      // the residual check and the fallback read it back
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int eh = e + h * NT;
+        bad |= !(isfinite(acc[h].x) && isfinite(acc[h].y) && isfinite(acc[h].z) && isfinite(acc[h].w));
+        *reinterpret_cast<float4*>(Gs + (eh / (D / 4)) * LD + (eh % (D / 4)) * 4) = acc[h];
+        reinterpret_cast<float4*>(gout)[eh] = acc[h];   // the residual check and the fallback read it back
+      }
     }
     if (tid < 4) s_flags[tid] = 0;
     if (tid == 0) s_why = 0;
@@ -234,147 +394,41 @@ eig_tridiag_kernel(const float* __restrict__ gpart, const int* __restrict__ gram
   int passes = 0;
   if (route != kRouteFull && gmax > 0.f) {
     // ---- 2. Householder tridiagonalisation, the matrix in registers ---------------------------
-    if (warp < TW) {
-      float a[RPL][D];
-      int rowq[RPL];
+    {
+      float a[RPT][CPT], xr[RPT], xc[CPT];
 #pragma unroll
-      for (int q = 0; q < RPL; ++q) {
-        rowq[q] = (TW == 1) ? lane + 32 * q : warp * 32 + lane;
+      for (int q = 0; q < RPT; ++q) {
 #pragma unroll
-        for (int jb = 0; jb < NB; ++jb) {
-          const float4 g = *reinterpret_cast<const float4*>(Gs + rowq[q] * LD + 4 * jb);
-          a[q][4 * jb] = g.x * sc; a[q][4 * jb + 1] = g.y * sc;
-          a[q][4 * jb + 2] = g.z * sc; a[q][4 * jb + 3] = g.w * sc;
+        for (int g = 0; g < NG; ++g) {
+          const float4 t = *reinterpret_cast<const float4*>(Gs + (lane + 32 * q) * LD + 4 * (warp + NW * g));
+          a[q][4 * g] = t.x * sc; a[q][4 * g + 1] = t.y * sc; a[q][4 * g + 2] = t.z * sc; a[q][4 * g + 3] = t.w * sc;
         }
+        xr[q] = Gs[(lane + 32 * q) * LD] * sc;                      // column 0 at my rows ...
       }
-      float xf[RPL];           // column k of the current matrix at my rows
 #pragma unroll
-      for (int q = 0; q < RPL; ++q) xf[q] = a[q][0];
-
-      for (int k = 0; k < D - 2; ++k) {
-        const int k1 = k + 1, jb0 = k1 >> 2, c1 = k1 & 3;
-        const bool skip0 = (RPL == 2) && (k >= 32);      // the lanes' first rows are all done
-        // x = column k below the subdiagonal; published as the reflector's vector (its element
-        // k+1 is patched in by the readers once alpha is known)
-        float xs[RPL], sq = 0.f;
-#pragma unroll
-        for (int q = 0; q < RPL; ++q) {
-          xs[q] = rowq[q] > k1 ? xf[q] : 0.f;
-          sq = fmaf(xs[q], xs[q], sq);
-          hv[k * D + rowq[q]] = xs[q];
-        }
-        float tail2, x1, dk;
-        if (TW == 1) {
-          float cand1 = xf[0], candk = xf[0];
-          if (RPL == 2) { cand1 = (k1 >= 32) ? xf[RPL - 1] : xf[0]; candk = (k >= 32) ? xf[RPL - 1] : xf[0]; }
-          x1 = __shfl_sync(kFull, cand1, k1 & 31);
-          dk = __shfl_sync(kFull, candk, k & 31);
-          tail2 = warp_sum(sq);
-          __syncwarp();
-        } else {
-          sq = warp_sum(sq);
-          if (lane == 0) s_red[0][warp] = sq;
-          if (rowq[0] == k1) s_scal[0] = xf[0];
-          if (rowq[0] == k) s_scal[1] = xf[0];
-          bar_named(1, TW * 32);
-          tail2 = (s_red[0][0] + s_red[0][1]) + (s_red[0][2] + s_red[0][3]);
-          x1 = s_scal[0]; dk = s_scal[1];
-        }
-        const bool reflect = tail2 > 1e-35f;               // uniform over the taking-part warps
-        float alpha = x1, beta = 0.f, vk1 = 0.f;
-        if (reflect) {
-          const float nrm = sqrtf(fmaf(x1, x1, tail2));
-          alpha = -copysignf(nrm, x1);
-          vk1 = x1 - alpha;
-          beta = 1.f / (nrm * (nrm + fabsf(x1)));
-        }
-        if (tid == 0) { dg[k] = dk; eo[k] = alpha; betas[k] = beta; }
-        if (!reflect) {
-          // nothing to annihilate: T takes the column as it is, the matrix stays
-#pragma unroll
-          for (int jb = 0; jb < NB; ++jb)
-            if (jb == jb0) {
-#pragma unroll
-              for (int q = 0; q < RPL; ++q)
-                xf[q] = c1 == 0 ? a[q][4 * jb] : c1 == 1 ? a[q][4 * jb + 1] : c1 == 2 ? a[q][4 * jb + 2] : a[q][4 * jb + 3];
-            }
-          if (TW > 1) bar_named(1, TW * 32);               // the exchange words are rewritten next step
-          continue;
-        }
-        float vi[RPL];
-#pragma unroll
-        for (int q = 0; q < RPL; ++q) {
-          vi[q] = (rowq[q] == k1) ? vk1 : xs[q];
-          if (rowq[q] == k1) hv[k * D + k1] = vk1;          // the complete vector, for step 5
-        }
-        // p = beta * A v over the trailing block (lane-local: a row against the broadcast v)
-        const float4* v4p = reinterpret_cast<const float4*>(hv + k * D);
-        float pa[RPL][2];
-#pragma unroll
-        for (int q = 0; q < RPL; ++q) { pa[q][0] = 0.f; pa[q][1] = 0.f; }
-#pragma unroll
-        for (int jb = 0; jb < NB; ++jb)
-          if (jb >= jb0) {
-            float4 v4 = v4p[jb];
-            if (jb == jb0) put4(v4, c1, vk1);
-#pragma unroll
-            for (int q = 0; q < RPL; ++q) {
-              if (q == 0 && skip0) continue;
-              float acc = pa[q][jb & 1];
-              acc = fmaf(a[q][4 * jb], v4.x, acc);     acc = fmaf(a[q][4 * jb + 1], v4.y, acc);
-              acc = fmaf(a[q][4 * jb + 2], v4.z, acc); acc = fmaf(a[q][4 * jb + 3], v4.w, acc);
-              pa[q][jb & 1] = acc;
-            }
-          }
-        float pi[RPL], pv = 0.f;
-#pragma unroll
-        for (int q = 0; q < RPL; ++q) {
-          pi[q] = rowq[q] > k ? beta * (pa[q][0] + pa[q][1]) : 0.f;
-          pv = fmaf(pi[q], vi[q], pv);
-        }
-        if (TW == 1) {
-          pv = warp_sum(pv);
-        } else {
-          pv = warp_sum(pv);
-          if (lane == 0) s_red[1][warp] = pv;
-          bar_named(1, TW * 32);
-          pv = (s_red[1][0] + s_red[1][1]) + (s_red[1][2] + s_red[1][3]);
-        }
-        const float kk = 0.5f * beta * pv;
-        float wi[RPL];
-#pragma unroll
-        for (int q = 0; q < RPL; ++q) {
-          wi[q] = fmaf(-kk, vi[q], pi[q]);
-          wv[rowq[q]] = wi[q];
-        }
-        if (TW == 1) __syncwarp(); else bar_named(1, TW * 32);
-        // A <- A - v w^T - w v^T on the trailing block; the first block touched holds column k+1
-        const float4* w4p = reinterpret_cast<const float4*>(wv);
-#pragma unroll
-        for (int jb = 0; jb < NB; ++jb)
-          if (jb >= jb0) {
-            float4 v4 = v4p[jb];
-            if (jb == jb0) put4(v4, c1, vk1);
-            const float4 w4 = w4p[jb];
-#pragma unroll
-            for (int q = 0; q < RPL; ++q) {
-              if (q == 0 && skip0) continue;
-              a[q][4 * jb]     = fmaf(-vi[q], w4.x, fmaf(-wi[q], v4.x, a[q][4 * jb]));
-              a[q][4 * jb + 1] = fmaf(-vi[q], w4.y, fmaf(-wi[q], v4.y, a[q][4 * jb + 1]));
-              a[q][4 * jb + 2] = fmaf(-vi[q], w4.z, fmaf(-wi[q], v4.z, a[q][4 * jb + 2]));
-              a[q][4 * jb + 3] = fmaf(-vi[q], w4.w, fmaf(-wi[q], v4.w, a[q][4 * jb + 3]));
-              if (jb == jb0)
-                xf[q] = c1 == 0 ? a[q][4 * jb] : c1 == 1 ? a[q][4 * jb + 1] : c1 == 2 ? a[q][4 * jb + 2] : a[q][4 * jb + 3];
-            }
-          }
+      for (int g = 0; g < NG; ++g) {
+        const float4 t = *reinterpret_cast<const float4*>(Gs + 4 * (warp + NW * g));   // ... and (row 0) at my columns
+        xc[4 * g] = t.x * sc; xc[4 * g + 1] = t.y * sc; xc[4 * g + 2] = t.z * sc; xc[4 * g + 3] = t.w * sc;
       }
-      // the last 2 x 2 block: xf holds column D-2
-#pragma unroll
-      for (int q = 0; q < RPL; ++q) {
-        if (rowq[q] == D - 2) dg[D - 2] = xf[q];
-        if (rowq[q] == D - 1) { eo[D - 2] = xf[q]; dg[D - 1] = a[q][D - 1]; }
+      for (int e = tid; e < D * D / 4; e += NT) reinterpret_cast<float4*>(hv)[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int e = tid; e < 2 * D; e += NT) xpre[e] = 0.f;
+      __syncthreads();
+      tri_stage<D, 0>(a, xr, xc, hv, xpre, tpart, pvp, dg, eo, betas, tid);
+      tri_stage<D, 1>(a, xr, xc, hv, xpre, tpart, pvp, dg, eo, betas, tid);
+      if constexpr (NG > 2) {
+        tri_stage<D, 2>(a, xr, xc, hv, xpre, tpart, pvp, dg, eo, betas, tid);
+        tri_stage<D, 3>(a, xr, xc, hv, xpre, tpart, pvp, dg, eo, betas, tid);
       }
-      if (tid == 0) { eo[D - 1] = 0.f; betas[D - 2] = 0.f; betas[D - 1] = 0.f; }
+      // the last 2 x 2 block: xr holds column D-2
+      if (warp == 0) {
+#pragma unroll
+        for (int q = 0; q < RPT; ++q) {
+          if (lane + 32 * q == D - 2) dg[D - 2] = xr[q];
+          if (lane + 32 * q == D - 1) eo[D - 2] = xr[q];
+        }
+        if (lane == 0) { eo[D - 1] = 0.f; betas[D - 2] = 0.f; betas[D - 1] = 0.f; }
+      }
+      if (warp == NW - 1 && lane == 31) dg[D - 1] = a[RPT - 1][CPT - 1];
     }
     __syncthreads();
 
@@ -397,99 +451,199 @@ eig_tridiag_kernel(const float* __restrict__ gpart, const int* __restrict__ gram
     }
     __syncthreads();
     const float tnorm = fmaxf(fabsf(s_lo), fabsf(s_hi));
-    if (warp < NE) {
-      const int j = warp * 32 + lane, jj = j < r ? j : r - 1;
+    // Eigenvalue j = 32 * gi + lane belongs to the group gi of WG warps; every warp of the group
+    // keeps the same bracket and evaluates its own interior point(s) in each step.
+    const int gi = warp / WG, wg = warp % WG;
+    const int j = gi * 32 + lane, jj = j < r ? j : r - 1;       // surplus lanes shadow column r-1
+    float lam;
+    {
+      constexpr int CH = (WG >= 4) ? 1 : 2;                      // points per warp and step
+      constexpr int P = CH * WG;                                 // 4 or 8 points: 5 or 9 sub-intervals
+      constexpr int STEPS = (P >= 8) ? 9 : 12;                   // (P + 1)^STEPS >= 2^27
+      static_assert(2 * NE * P * 32 <= RP * RP, "flags fit in the E region");
+      unsigned char* flag = reinterpret_cast<unsigned char*>(Em);   // [2][NE][P][32]: count(point) > target
       const int target = D - 1 - jj;      // lambda_(jj-th largest) >= x  <=>  #(eigenvalues < x) <= target
       float lo = s_lo, hi = s_hi;
 #pragma unroll 1
-      for (int step = 0; step < 13; ++step) {
-        const float w = hi - lo;
-        const float m1 = fmaf(0.25f, w, lo), m2 = fmaf(0.5f, w, lo), m3 = fmaf(0.75f, w, lo);
-        int c1, c2, c3;
-        sturm3<D>(dg, e2s, m1, m2, m3, c1, c2, c3);
-        if (c1 > target) { hi = m1; }
-        else if (c2 > target) { lo = m1; hi = m2; }
-        else if (c3 > target) { lo = m2; hi = m3; }
-        else { lo = m3; }
+      for (int step = 0; step < STEPS; ++step) {
+        const float w = (hi - lo) * (1.f / (P + 1));
+        float x[CH];
+        int cnt[CH];
+#pragma unroll
+        for (int h = 0; h < CH; ++h) x[h] = fmaf((float)(wg * CH + h + 1), w, lo);
+        sturm<D, CH>(dg, e2s, x, cnt);
+        unsigned char* fl = flag + (((step & 1) * NE + gi) * P) * 32;
+#pragma unroll
+        for (int h = 0; h < CH; ++h) fl[(wg * CH + h) * 32 + lane] = cnt[h] > target;
+        __syncthreads();
+        int idx = P;                       // first point above the eigenvalue
+#pragma unroll
+        for (int pnt = P - 1; pnt >= 0; --pnt) idx = fl[pnt * 32 + lane] ? pnt : idx;
+        const float nlo = idx == 0 ? lo : fmaf((float)idx, w, lo);
+        const float nhi = idx == P ? hi : fmaf((float)(idx + 1), w, lo);
+        lo = nlo; hi = nhi;
       }
-      const float lam = 0.5f * (lo + hi);
-      lamv[j] = lam;
+      lam = 0.5f * (lo + hi);
+      if (wg == 0) lamv[j] = lam;
+    }
 
-      // ---- 4. twisted factorisation: one vector per lane -----------------------------------------
-      float* tf = work;                 // [D][RP] forward pivots, then the upward multipliers
-      float* tb = work + D * RP;        // [D][RP] backward pivots, then the downward multipliers
-      const float pfl = tnorm * 9.3132257e-10f;                              // pivot floor 2^-30 |T|
-      {
-        float qf = dg[0] - lam, qb = dg[D - 1] - lam;
-        qf = fabsf(qf) < pfl ? -pfl : qf; qb = fabsf(qb) < pfl ? -pfl : qb;
-        tf[j] = qf; tb[(D - 1) * RP + j] = qb;
-#pragma unroll 4
-        for (int t = 1; t < D; ++t) {
+    // ---- 4. twisted factorisation ---------------------------------------------------------------
+    // The pivots of the two triangular factorisations of T - lambda I are ratios of consecutive
+    // minors: q+_i = p_{i+1} / p_i with the leading minors p of the Sturm recurrence, and
+    // q-_i = t_i / t_{i+1} with the trailing minors t.  Taking them from the (rescaled) minor
+    // recurrences keeps the divisions off the dependency chain, which is one FMA per step.  The
+    // forward and the backward sequence run on two warps of the group; then every warp takes a
+    // range of i for gamma_i and the multipliers; then two warps run the two halves of z.
+    float* tf = work;                 // [D][RP] forward pivots, then the upward multipliers / values
+    float* tb = work + D * RP;        // [D][RP] backward pivots, then the downward multipliers / values
+    const float pfl = tnorm * 9.3132257e-10f;                                // pivot floor 2^-30 |T|
+    constexpr int WB = (WG > 1) ? 1 : 0;                                     // the warp of the backward sequences
+    {
+      if (wg == 0) {
+        float pf = 1.f, pfo = 0.f;                              // p_i, p_{i-1}
+#pragma unroll 8
+        for (int t = 0; t < D; ++t) {
+          const float nf = fmaf(dg[t] - lam, pf, -(e2s[t] * pfo));
+          float qf = __fdividef(nf, pf);
+          qf = (fabsf(qf) >= pfl) ? qf : -pfl;                   // also catches NaN
+          tf[t * RP + j] = qf;
+          pfo = pf; pf = nf;
+          if ((t & 3) == 3) {
+            const unsigned mf = __float_as_uint(fmaxf(fabsf(pf), fabsf(pfo))) >> 23;
+            const float sf = __uint_as_float((254u - mf) << 23);
+            pf *= sf; pfo *= sf;
+          }
+        }
+      }
+      if (wg == WB) {
+        float pb = 1.f, pbo = 0.f;                              // t_{i+1}, t_{i+2}
+#pragma unroll 8
+        for (int t = 0; t < D; ++t) {
           const int ib = D - 1 - t;
-          qf = (dg[t] - lam) - __fdividef(e2s[t], qf);
-          qb = (dg[ib] - lam) - __fdividef(e2s[ib + 1], qb);
-          qf = fabsf(qf) < pfl ? -pfl : qf; qb = fabsf(qb) < pfl ? -pfl : qb;
-          tf[t * RP + j] = qf; tb[ib * RP + j] = qb;
+          const float nb = fmaf(dg[ib] - lam, pb, -((t > 0 ? e2s[ib + 1] : 0.f) * pbo));
+          float qb = __fdividef(nb, pb);
+          qb = (fabsf(qb) >= pfl) ? qb : -pfl;
+          tb[ib * RP + j] = qb;
+          pbo = pb; pb = nb;
+          if ((t & 3) == 3) {
+            const unsigned mb = __float_as_uint(fmaxf(fabsf(pb), fabsf(pbo))) >> 23;
+            const float sb = __uint_as_float((254u - mb) << 23);
+            pb *= sb; pbo *= sb;
+          }
         }
       }
-      int kt = 0;
-      {
-        float best = 3.0e38f;
-#pragma unroll 4
-        for (int i = 0; i < D; ++i) {
-          const float qf = tf[i * RP + j], qb = tb[i * RP + j];
-          const float gam = fabsf((qf + qb) - (dg[i] - lam));
-          if (gam < best) { best = gam; kt = i; }
-          // z_i = -(e_i / q+_i) z_{i+1} going up, z_i = -(e_{i-1} / q-_i) z_{i-1} going down
-          tf[i * RP + j] = -__fdividef(eo[i], qf);
-          tb[i * RP + j] = i > 0 ? -__fdividef(eo[i - 1], qb) : 0.f;
-        }
+    }
+    __syncthreads();
+    {
+      // gamma_i = q+_i + q-_i - (d_i - lambda) over my range of i; the multipliers
+      // z_i = -(e_i / q+_i) z_{i+1} going up, z_i = -(e_{i-1} / q-_i) z_{i-1} going down
+      constexpr int IR = D / WG;
+      float best = 3.0e38f;
+      int kb = 0;
+#pragma unroll 8
+      for (int i = wg * IR; i < (wg + 1) * IR; ++i) {
+        const float qf = tf[i * RP + j], qb = tb[i * RP + j];
+        const float gam = fabsf((qf + qb) - (dg[i] - lam));
+        if (gam < best) { best = gam; kb = i; }
+        tf[i * RP + j] = -__fdividef(eo[i], qf);
+        tb[i * RP + j] = i > 0 ? -__fdividef(eo[i - 1], qb) : 0.f;
       }
-      float ss = 1.f;
-      {
-        float zu = 1.f, zd = 1.f;
-#pragma unroll 4
+      part[wg * RP + j] = best;
+      reinterpret_cast<int*>(part)[(NW + wg) * RP + j] = kb;
+    }
+    __syncthreads();
+    int kt = 0;
+    {
+      float best = 3.0e38f;
+#pragma unroll
+      for (int w2 = 0; w2 < WG; ++w2) {
+        const float bv = part[w2 * RP + j];
+        const int bk = reinterpret_cast<const int*>(part)[(NW + w2) * RP + j];
+        if (bv < best) { best = bv; kt = bk; }                   // ranges ascend: the lowest i wins a tie
+      }
+    }
+    __syncthreads();
+    {
+      // z_kt = 1; the values above the twist overwrite tf, those below it tb (no branches: a lane
+      // that has not reached its twist index yet keeps z = 1)
+      if (wg == 0) {
+        float zu = 1.f, ss = 0.f;
+#pragma unroll 8
+        for (int iu = D - 2; iu >= 0; --iu) {
+          const float mu = tf[iu * RP + j];
+          zu = (iu < kt) ? zu * mu : 1.f;
+          ss = fmaf(zu, (iu < kt) ? zu : 0.f, ss);
+          tf[iu * RP + j] = zu;
+        }
+        part[j] = ss;
+        ktv[j] = kt;
+      }
+      if (wg == WB) {
+        float zd = 1.f, ss = 0.f;
+#pragma unroll 8
         for (int t = 1; t < D; ++t) {
-          const int iu = D - 1 - t;            // upward: D-2 .. 0;  downward: 1 .. D-1
-          const float mu = tf[iu * RP + j], md = tb[t * RP + j];
-          if (iu < kt) { zu *= mu; ss = fmaf(zu, zu, ss); }
-          if (t > kt) { zd *= md; ss = fmaf(zd, zd, ss); }
-          if (iu < kt) vs[iu * RP + j] = zu;
-          if (t > kt) vs[t * RP + j] = zd;
+          const float md = tb[t * RP + j];
+          zd = (t > kt) ? zd * md : 1.f;
+          ss = fmaf(zd, (t > kt) ? zd : 0.f, ss);
+          tb[t * RP + j] = zd;
         }
-        vs[kt * RP + j] = 1.f;
+        part[RP + j] = ss;
       }
-      const float zn = rsqrtf(ss);
+    }
+    __syncthreads();
+    if (wg == 0) sgn[j] = rsqrtf(1.f + part[j] + part[RP + j]);   // 1 / |z|
+    __syncthreads();
 
-      // ---- 5. back-transformation: v = H_0 H_1 ... H_{D-3} z, the vector in registers -------------
-      float z[D];
-#pragma unroll
-      for (int i = 0; i < D; ++i) z[i] = vs[i * RP + j] * zn;
+    // ---- 5. back-transformation: v = H_0 H_1 ... H_{D-3} z ------------------------------------
+    // Four threads per vector, each with a quarter of the rows in registers; the reflector's
+    // inner product is completed by two shuffles.  Reflector k is zero at rows <= k, so the
+    // quarters need no conditions.
+    {
+      constexpr int RB = D / 4;                   // rows per thread
+      constexpr int VPP = NT / 4;                 // vectors per pass
+      constexpr int NPASS = (RP + VPP - 1) / VPP;
+      static_assert(NPASS * VPP >= RP, "every vector is transformed");
 #pragma unroll 1
-      for (int k = D - 3; k >= 0; --k) {
-        const float beta = betas[k];
-        if (beta == 0.f) continue;                      // uniform
-        const int ib0 = (k + 1) >> 2;                   // rows <= k of reflector k are zero
-        const float4* h4 = reinterpret_cast<const float4*>(hv + k * D);
-        float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
+      for (int pass = 0; pass < NPASS; ++pass) {
+        const int jv = pass * VPP + (tid >> 2), qt = tid & 3;
+        const bool act = jv < RP;
+        const int jc = act ? jv : 0;
+        const int ktj = ktv[jc];
+        const float zn = sgn[jc];
+        float z[RB];
 #pragma unroll
-        for (int ib = 0; ib < NB; ++ib)
-          if (ib >= ib0) {
-            const float4 h = h4[ib];
-            d0 = fmaf(h.x, z[4 * ib], d0); d1 = fmaf(h.y, z[4 * ib + 1], d1);
-            d2 = fmaf(h.z, z[4 * ib + 2], d2); d3 = fmaf(h.w, z[4 * ib + 3], d3);
-          }
-        const float c = -beta * ((d0 + d1) + (d2 + d3));
+        for (int u = 0; u < RB; ++u) {
+          const int i = qt * RB + u;
+          const float upv = tf[i * RP + jc], dnv = tb[i * RP + jc];
+          z[u] = (i < ktj ? upv : i > ktj ? dnv : 1.f) * zn;
+        }
+#pragma unroll 2
+        for (int k = D - 3; k >= 0; --k) {
+          const float beta = betas[k];
+          const float4* h4 = reinterpret_cast<const float4*>(hv + k * D + qt * RB);
+          float4 h[RB / 4];
+          float d0 = 0.f, d1 = 0.f;
 #pragma unroll
-        for (int ib = 0; ib < NB; ++ib)
-          if (ib >= ib0) {
-            const float4 h = h4[ib];
-            z[4 * ib] = fmaf(c, h.x, z[4 * ib]);         z[4 * ib + 1] = fmaf(c, h.y, z[4 * ib + 1]);
-            z[4 * ib + 2] = fmaf(c, h.z, z[4 * ib + 2]); z[4 * ib + 3] = fmaf(c, h.w, z[4 * ib + 3]);
+          for (int u = 0; u < RB / 4; ++u) {
+            h[u] = h4[u];
+            d0 = fmaf(h[u].x, z[4 * u], d0);     d1 = fmaf(h[u].y, z[4 * u + 1], d1);
+            d0 = fmaf(h[u].z, z[4 * u + 2], d0); d1 = fmaf(h[u].w, z[4 * u + 3], d1);
           }
+          float dt = d0 + d1;
+          dt += __shfl_xor_sync(kFull, dt, 1);
+          dt += __shfl_xor_sync(kFull, dt, 2);
+          const float c = -beta * dt;
+#pragma unroll
+          for (int u = 0; u < RB / 4; ++u) {
+            z[4 * u] = fmaf(c, h[u].x, z[4 * u]);         z[4 * u + 1] = fmaf(c, h[u].y, z[4 * u + 1]);
+            z[4 * u + 2] = fmaf(c, h[u].z, z[4 * u + 2]); z[4 * u + 3] = fmaf(c, h[u].w, z[4 * u + 3]);
+          }
+        }
+        if (act) {
+#pragma unroll
+          for (int u = 0; u < RB; ++u) vs[(qt * RB + u) * RP + jv] = z[u];
+        }
       }
-#pragma unroll
-      for (int i = 0; i < D; ++i) vs[i * RP + j] = z[i];
     }
     __syncthreads();
     pdl_trigger();     // the long serial part is over: the next kernel may start launching
@@ -514,7 +668,7 @@ eig_tridiag_kernel(const float* __restrict__ gpart, const int* __restrict__ gram
 #pragma unroll
         for (int u = 0; u < AW; ++u) acc[h][u] = 0.f;
       const int a0 = warp * AW;
-#pragma unroll 2
+#pragma unroll 8
       for (int i = 0; i < D; ++i) {
         float av[AW];
         if (AW >= 4) {
@@ -595,7 +749,7 @@ eig_tridiag_kernel(const float* __restrict__ gpart, const int* __restrict__ gram
 #pragma unroll
         for (int u = 0; u < RW; ++u) y[h][u] = 0.f;
       const int i0 = warp * RW;
-#pragma unroll 1
+#pragma unroll 2
       for (int k = 0; k < D; k += 4) {
         float vk[NE][4];
 #pragma unroll
