@@ -2,17 +2,22 @@
 """Benchmark of the SVD-Attention forward pass (solar_lowrank_factor + solar_svd_attention_fwd).
 
 One "step" = one pass of the whole hot path over one batch of B users: streaming Gram of
-H, Jacobi eigensolve, factor-token projections, candidate attention.  Metric: candidates x
+H, eigensolve, factor-token projections, candidate attention.  Metric: candidates x
 sequence positions per second = B*M*N / step time.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3] [--in-flight S]
-                    [--impl ours|reference]
+                    [--path fused|two_call] [--impl ours|reference]
 
 The timed region replays CUDA graphs of whole steps (no host work between kernels).  With
 --in-flight S > 1, S independent batches are in flight on S streams (each with its own
 workspace and factors), which is how a serving process overlaps one request's eigensolve
-(16 CTAs) with another's streaming passes; S = 1 gives the single-call latency.  Both
-figures are printed; `value` is the one at the S given (default 16).
+(B CTAs) with another's streaming passes; S = 1 gives the single-call latency.  Both
+figures are printed; `value` is the one at the S given (default 24).  Every step in flight
+reads and writes buffers of its own (2 S + 7 buffer sets), --steps is a minimum, and the
+timed region lasts at least half a second; the spread over the graph replays is printed.
+`value` is measured through solar_svd_attention_fused (three launches per step); the same
+measurement through solar_lowrank_factor + solar_svd_attention_fwd (four launches) is
+printed beside it as `two_call`.
 
 Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs its own batches of B
 users (users are independent: no data-path collective), timing is max over ranks.
@@ -37,7 +42,7 @@ from paper_2603_02561_b200 import bench_plan as bp  # noqa: E402
 from paper_2603_02561_b200 import workloads as wl  # noqa: E402
 
 L2_BYTES = 126 * 2 ** 20
-KERNELS_PER_STEP = 4          # gram, eigensolve, factor-token projections, attention
+KERNELS_PER_STEP = {"fused": 3, "two_call": 4}   # gram, eigensolve (+ projections), [projections,] attention
 FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # 148 SMs x 128 FMA lanes x 2 flop at 1965 MHz
 SFU_TEXPS = 148 * 16 * 1.965e9 / 1e12              # 148 SMs x 16 special-function lanes at 1965 MHz
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
@@ -178,14 +183,21 @@ def run_reference(args, w: wl.Workload):
 
 
 # ---------------------------------------------------------------------------------------
-def eig_flops(w: wl.Workload, iters: float, sweeps: float, route_full: bool) -> float:
-    """Useful floating-point operations of the eigensolver for one batch (both routes counted
-    from their loop bounds: dense products 2mnk, a 2x2 Jacobi block update 24 flop for the
-    matrix and 12 for the vectors)."""
-    d = w.d
-    if route_full:
+def eig_flops(w: wl.Workload, route: int, detail: float, sweeps: float) -> float:
+    """Useful floating-point operations of the eigensolver for one batch, counted from loop
+    bounds.  Route 3 (tridiagonal): reduction 4/3 d^3, back-transformation 2 d^2 r, each
+    orthogonalisation pass 4 d r^2, residuals 2 d^2 r, multisection 3 d r per point and step
+    (26 bits), twisted factorisation ~20 d r.  Route 1 / 2 (range finder, Jacobi): dense
+    products 2mnk, a 2x2 Jacobi block update 24 flop for the matrix and 12 for the vectors."""
+    d, r = w.d, w.r
+    if route == 3:
+        passes = sweeps
+        return w.B * (4.0 * d ** 3 / 3 + 4.0 * d * d * r + (passes + 1) * 2.0 * d * r * r + passes * 2.0 * d * r * r
+                      + 3.0 * d * r * 4 * 12 + 20.0 * d * r)
+    if route == 2:
         return w.B * sweeps * (d - 1) * (d * d / 4) * 36.0
-    p = (w.r + 7) // 8 * 8
+    p = (r + 7) // 8 * 8
+    iters = detail
     power = (iters + 1) * 2 * d * d * p + iters * (2 * d * p * p + p ** 3 / 3 + 2 * d * p * p) + 2 * d * p * p
     jac = sweeps * (p - 1) * (p * p / 4) * 36.0
     return w.B * (power + jac + 4 * d * p * p)
@@ -198,7 +210,7 @@ class Lane:
         self.stream = torch.cuda.Stream()
         self.S = torch.empty(w.B, w.r, device="cuda")
         self.V = torch.empty(w.B, w.d, w.r, device="cuda")
-        self.ws = solar.alloc_workspace(w.B, w.M, w.N, w.d, w.r, tdt)
+        self.ws = solar.alloc_fused_workspace(w.B, w.M, w.N, w.d, w.r, tdt)   # covers the two-call sizes too
 
 
 def main():
@@ -209,6 +221,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3")
     ap.add_argument("--in-flight", type=int, default=24, help="independent batches in flight (streams)")
+    ap.add_argument("--path", default="fused", choices=["fused", "two_call"],
+                    help="which public call `value` is measured through (the other is printed beside it)")
     ap.add_argument("--cpu-users", type=int, default=8, help="users in the cpu_baseline sample")
     ap.add_argument("--ref-users", type=int, default=2, help="users per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -279,37 +293,49 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
     """Times workload w on this rank's GPU; returns the JSON line (rank 0) or None."""
     tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
     ab = algorithmic_bytes(w)
-    # rotate over enough distinct batches that a step's inputs are never L2-resident
-    nb = bp.batches_to_exceed_l2(ab["total"], L2_BYTES)
-    batches = [wl.generate(w.with_(seed_index=si)) for si in bp.rank_seed_indices(w.seed_index, rank, nb)]
+    # Distinct data: enough seeded batches that a step's inputs are never L2-resident.  Distinct
+    # BUFFERS: every step that can be in flight together with another reads and writes buffers of
+    # its own (2 x lanes + the L2 margin); buffers beyond the seeded batches hold device copies
+    # of them with the users rotated, which is all the DRAM traffic cares about.
+    n_lanes = max(1, args.in_flight)
+    nseed = bp.batches_to_exceed_l2(ab["total"], L2_BYTES)
+    nb = bp.distinct_buffers(n_lanes, nseed)
+    batches = [wl.generate(w.with_(seed_index=si)) for si in bp.rank_seed_indices(w.seed_index, rank, nseed)]
     Wq, Wk, Wv = (torch.from_numpy(batches[0][k]).cuda().to(tdt) for k in ("Wq", "Wk", "Wv"))
     dH = [torch.from_numpy(b["H"]).cuda().to(tdt) for b in batches]
     dC = [torch.from_numpy(b["C"]).cuda().to(tdt) for b in batches]
+    for k in range(nseed, nb):
+        dH.append(torch.roll(dH[k % nseed], 1 + k // nseed, 0).contiguous())
+        dC.append(torch.roll(dC[k % nseed], 1 + k // nseed, 0).contiguous())
     dO = [torch.empty_like(c) for c in dC]
     main_stream = torch.cuda.Stream()
-    n_lanes = max(1, args.in_flight)
     lanes = [Lane(torch, solar, w, tdt) for _ in range(n_lanes)]
 
-    def step(k, lane, stream):
-        solar.lowrank_factor(dH[k], w.r, S=lane.S, V=lane.V, workspace=lane.ws, M=w.M, stream=stream)
-        solar.svd_attention_fwd(dC[k], lane.S, lane.V, Wq, Wk, Wv, w.scale, 0, O=dO[k], workspace=lane.ws,
-                                N=w.N, stream=stream)
+    def step(k, lane, stream, path=None):
+        if (path or args.path) == "fused":
+            solar.svd_attention_fused(dH[k], dC[k], Wq, Wk, Wv, w.r, w.scale, 0, S=lane.S, V=lane.V, O=dO[k],
+                                      workspace=lane.ws, stream=stream)
+        else:
+            solar.lowrank_factor(dH[k], w.r, S=lane.S, V=lane.V, workspace=lane.ws, M=w.M, stream=stream)
+            solar.svd_attention_fwd(dC[k], lane.S, lane.V, Wq, Wk, Wv, w.scale, 0, O=dO[k], workspace=lane.ws,
+                                    N=w.N, stream=stream)
 
-    def capture(n_steps, use_lanes):
-        """A CUDA graph of n_steps whole steps, dealt round-robin to the lanes' streams."""
+    def capture(rounds, use_lanes, path=None):
+        """A CUDA graph of `rounds` whole steps on each of the lanes' streams."""
+        L = len(use_lanes)
         g = torch.cuda.CUDAGraph()
         with torch.cuda.stream(main_stream):
             with torch.cuda.graph(g, stream=main_stream, capture_error_mode="relaxed"):
-                if len(use_lanes) == 1:
-                    for i in range(n_steps):
-                        step(i % nb, use_lanes[0], main_stream)
+                if L == 1:
+                    for i in range(rounds):
+                        step(bp.buffer_of_step(i, 0, 1, nb), use_lanes[0], main_stream, path)
                 else:
                     fork = torch.cuda.Event()
                     fork.record(main_stream)
                     for li, lane in enumerate(use_lanes):
                         lane.stream.wait_event(fork)
-                        for i in range(li, n_steps, len(use_lanes)):
-                            step(i % nb, lane, lane.stream)
+                        for i in range(rounds):
+                            step(bp.buffer_of_step(i, li, L, nb), lane, lane.stream, path)
                         join = torch.cuda.Event()
                         join.record(lane.stream)
                         main_stream.wait_event(join)
@@ -321,41 +347,79 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
         torch.cuda.synchronize()
 
     def timed_replays(g, n):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        """n replays back to back; an event after each, so the spread over replays is known."""
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
         with torch.cuda.stream(main_stream):
-            e0.record(main_stream)
-            for _ in range(n):
+            ev[0].record(main_stream)
+            for i in range(n):
                 g.replay()
-            e1.record(main_stream)
-        return e0, e1
+                ev[i + 1].record(main_stream)
+        return ev
+
+    def per_replay_ms(ev):
+        return [ev[i].elapsed_time(ev[i + 1]) for i in range(len(ev) - 1)]
 
     # the first call on a device sets kernel attributes: keep it outside any capture
-    for lane in lanes:
-        step(0, lane, main_stream)
+    for lane in lanes[:2]:
+        for path in ("fused", "two_call"):
+            step(0, lane, main_stream, path)
     torch.cuda.synchronize()
 
-    steps_per_graph, replays, steps = bp.replay_plan(args.steps, nb, n_lanes)
-    g_main = capture(steps_per_graph, lanes)
+    ROUNDS = 12
+    other = "two_call" if args.path == "fused" else "fused"
+    g_main = capture(ROUNDS, lanes)
+    g_other = capture(ROUNDS, lanes, other) if not light else None
     g_single = capture(nb, lanes[:1]) if n_lanes > 1 else g_main
-    warm = max(1, -(-max(args.warmup, 3) // steps_per_graph))
+    # warm-up (at least 3 steps and the --warmup asked for), which also calibrates the plan
+    warm = max(1, -(-max(args.warmup, 3) // (ROUNDS * n_lanes)))
     with torch.cuda.stream(main_stream):
         for _ in range(warm):
             g_main.replay()
             g_single.replay()
+            if g_other is not None:
+                g_other.replay()
     sync_all()
+    cal = timed_replays(g_main, 2)
+    sync_all()
+    est_ms = min(per_replay_ms(cal)) / (ROUNDS * n_lanes)
+    steps_per_graph, replays, steps = bp.replay_plan(args.steps, n_lanes, est_ms, rounds_per_graph=ROUNDS,
+                                                     min_seconds=0.1 if light else 0.5,
+                                                     min_replays=10 if light else 50)
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
     sync_all()
-    e0, e1 = timed_replays(g_main, replays)
+    ev = timed_replays(g_main, replays)
     sync_all()
-    ms = e0.elapsed_time(e1)
+    ms = ev[0].elapsed_time(ev[-1])
+    spread_main = bp.spread(per_replay_ms(ev), steps_per_graph)
+    ms_other, spread_other = None, None
+    if g_other is not None:
+        evo = timed_replays(g_other, max(10, replays // 4))
+        sync_all()
+        ms_other = evo[0].elapsed_time(evo[-1]) / ((len(evo) - 1) * steps_per_graph)
+        spread_other = bp.spread(per_replay_ms(evo), steps_per_graph)
     # single-call latency: one step at a time on one stream
     single_reps = max(3, min(replays * steps_per_graph // nb, 100))
-    s0, s1 = timed_replays(g_single, single_reps)
+    sev = timed_replays(g_single, single_reps)
     sync_all()
-    ms_single = s0.elapsed_time(s1) / (single_reps * nb)
+    ms_single = sev[0].elapsed_time(sev[-1]) / (single_reps * (nb if n_lanes > 1 else steps_per_graph))
+    # ... and as plain calls (no graph): what a caller without graphs pays per step, host work included
+    plain_n = 50
+    for _ in range(5):
+        step(0, lanes[0], main_stream)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(plain_n):
+        step(i % nb, lanes[0], main_stream)
+    torch.cuda.synchronize()
+    ms_plain = (time.perf_counter() - t0) * 1e3 / plain_n
+
+    def timed_graph_ms(g, reps):
+        e = timed_replays(g, reps)
+        torch.cuda.synchronize()
+        return e[0].elapsed_time(e[-1])
 
     # per-stage timing: each kernel alone, nb launches (rotating batches) per graph replay
     lane0 = lanes[0]
@@ -391,9 +455,7 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
                 g.replay()
         torch.cuda.synchronize()
         reps = 20
-        a, b = timed_replays(g, reps)
-        torch.cuda.synchronize()
-        stage_ms[name] = a.elapsed_time(b) / (reps * nb)
+        stage_ms[name] = timed_graph_ms(g, reps) / (reps * nb)
         if name == "eig":
             route_words = taken.cpu().numpy()
     # the factored-exact softmax attention over the N positions (beside the hot path, not part
@@ -416,9 +478,7 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
                                                          workspace=lane0.ws, stream=main_stream)
             g.replay()
         torch.cuda.synchronize()
-        a, b = timed_replays(g, 5)
-        torch.cuda.synchronize()
-        f_ms = a.elapsed_time(b) / (5 * nb)
+        f_ms = timed_graph_ms(g, 5) / (5 * nb)
         exps = float(w.pairs)
         factored = {"ms_per_call": f_ms, "value": w.pairs / (f_ms * 1e-3), "unit": "pairs/s",
                     "what": "solar_factored_softmax_attention_fwd (operand set-up + flash kernel), US resident",
@@ -431,12 +491,12 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
     if not light:
         bws = solar.alloc_backward_workspace(w.B, w.M, w.N, w.d, w.r, tdt)
         dHg = torch.empty_like(dH[0])
-        gO = [torch.randn(w.B, w.M, w.d, device="cuda").to(tdt) for _ in range(nb)]
+        gO = [torch.randn(w.B, w.M, w.d, device="cuda").to(tdt) for _ in range(min(nb, 8))]
         grads = solar.alloc_attention_grads(dC[0], w.r)
 
         def bwd_part(k, which):
             if which in (0, 2):
-                solar.svd_attention_bwd(dC[k], lane0.S, lane0.V, Wq, Wk, Wv, w.scale, gO[k], bws, out=grads,
+                solar.svd_attention_bwd(dC[k], lane0.S, lane0.V, Wq, Wk, Wv, w.scale, gO[k % len(gO)], bws, out=grads,
                                         stream=main_stream)
             if which in (1, 2):
                 solar.svd_backward(dH[k], lane0.S, lane0.V, grads[4], grads[5], dHg, bws, stream=main_stream)
@@ -454,9 +514,7 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
                         bwd_part(k, which)
                 g.replay()
             torch.cuda.synchronize()
-            a, b = timed_replays(g, 5)
-            torch.cuda.synchronize()
-            b_ms.append(a.elapsed_time(b) / (5 * nb))
+            b_ms.append(timed_graph_ms(g, 5) / (5 * nb))
         es = 2 if w.dtype == "bf16" else 4
         bwd_bytes = es * w.B * (3 * w.M * w.d + 2 * w.N * w.d)        # C, dO, dC; H, dH
         backward = {"ms_per_call": b_ms[2], "attention_bwd_ms": b_ms[0], "svd_backward_ms": b_ms[1],
@@ -512,7 +570,7 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
     routes = sorted(set(int(x) & 0xFF for x in route_words))
     iters = float(np.mean([(int(x) >> 8) & 0xFF for x in route_words]))
     sweeps = float(np.mean([(int(x) >> 16) & 0xFF for x in route_words]))
-    eflops = eig_flops(w, iters, sweeps, route_full=(routes == [2]))
+    eflops = eig_flops(w, max(routes), iters, sweeps)
     per_kernel = {
         "gram": {"bound": "hbm", "achieved": ab["gram"] / (stage_ms["gram"] * 1e-3) / 1e9, "peak": pk["hbm_gbs"],
                  "unit": "GB/s"},
@@ -530,14 +588,26 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
     line = {
         "metric": "svd_attention_fwd_candidates_x_positions_per_sec",
         "value": value, "unit": "pairs/s", "n_gpus": world, "steps": steps,
-        "warmup": warm * steps_per_graph, "ms_per_step": ms_step, "higher_is_better": True,
+        "warmup": warm * steps_per_graph + 2 * steps_per_graph, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "N": w.N, "d": w.d, "r": w.r, "M": w.M,
-                   "storage": w.dtype, "users_per_gpu": w.B, "in_flight": n_lanes,
-                   "launch": f"CUDA graphs of {steps_per_graph} steps, {replays} replays",
-                   "l2": f"inputs rotate over {nb} distinct batches ({nb * ab['total'] / 2**20:.0f} MiB > 126 MiB L2)"},
+                   "storage": w.dtype, "users_per_gpu": w.B, "in_flight": n_lanes, "path": args.path,
+                   "launch": f"CUDA graphs of {steps_per_graph} steps ({ROUNDS} per lane), {replays} replays, "
+                             f"{ms * 1e-3:.2f} s timed",
+                   "distinct_batches": nb, "seeded_batches": nseed,
+                   "l2": f"every step in flight has its own input and output buffers: {nb} buffer sets "
+                         f"({nb * ab['total'] / 2**20:.0f} MiB > 126 MiB L2), {nseed} seeded batches and device "
+                         "copies of them with the users rotated"},
+        "ms_per_step_spread": spread_main,
         "single_call": {"ms_per_step": ms_single, "value": world * w.pairs / (ms_single * 1e-3),
-                        "note": "one step at a time on one stream (in_flight = 1)"},
+                        "note": "one step at a time on one stream (in_flight = 1), graph replay",
+                        "plain_calls_ms_per_step": ms_plain,
+                        "plain_calls_note": "the same without a graph: host launch work included"},
+        ("two_call" if args.path == "fused" else "fused"): (None if ms_other is None else {
+            "ms_per_step": ms_other, "value": world * w.pairs / (ms_other * 1e-3), "spread": spread_other,
+            "frac": (w.pairs / (ms_other * 1e-3)) / (w.pairs / roof_s),
+            "what": ("solar_lowrank_factor + solar_svd_attention_fwd (four launches per step)"
+                     if args.path == "fused" else "solar_svd_attention_fused (three launches per step)")}),
         "path_roofline": {"bound": "hbm", "algorithmic_bytes": ab["total"],
                           "algorithmic_flops": algorithmic_flops(w),
                           "roofline_pairs_per_s": w.pairs / roof_s, "frac": value / world / (w.pairs / roof_s),
@@ -547,8 +617,9 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
         "roofline_by_kernel": per_kernel,
         "stage_ms": stage_ms, "stage_share": {k: v / tot for k, v in stage_ms.items()},
         "dominant_stage": dominant,
-        "eig_route": {"routes": routes, "power_steps": iters, "jacobi_sweeps": sweeps},
-        "gpu_launches": KERNELS_PER_STEP * steps,
+        "eig_route": {"routes": routes, "power_steps": iters, "sweeps_or_passes": sweeps,
+                      "note": "route 3 = tridiagonal (orthogonalisation passes), 2 = Jacobi (sweeps), 1 = range finder"},
+        "gpu_launches": KERNELS_PER_STEP[args.path] * steps,
         "clocks": clocks,
         "factored_exact": factored,
         "backward": backward,

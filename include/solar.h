@@ -13,7 +13,9 @@
  *     H, C, W_Q, W_K, W_V, O and US.  Arithmetic accumulates in fp32 (or wider).
  *   - Every pointer is a DEVICE pointer owned by the caller, 16-byte aligned,
  *     valid until the work queued on `stream` has finished.  The library
- *     allocates nothing and keeps no state between calls.
+ *     allocates nothing and keeps no state between calls.  Inputs may be written
+ *     by work queued earlier on the same stream: the first kernel of every call
+ *     waits for that work to complete before it reads any caller buffer.
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL =
  *     the legacy default stream) and never synchronise.
  *   - Errors the host can see (bad sizes, NULL or misaligned pointers, a
@@ -136,6 +138,25 @@ solar_status_t solar_svd_attention_fwd(int B, int M, int N, int d, int r, solar_
                                        const void* Wq, const void* Wk, const void* Wv,
                                        float scale, unsigned flags, void* O,
                                        void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The whole forward pass in one call: solar_lowrank_factor followed by
+ * solar_svd_attention_fwd (Eq. 9-12), with the same arguments, outputs, info bits and
+ * rules, and the same bits in S, V and O.  Three launches instead of four: every user's
+ * eigensolver CTA ends with that user's factor-token projections (Eq. 11), so the
+ * stand-alone projection kernel and its launch disappear.  S and V are still written.
+ *
+ *   workspace: solar_fused_workspace_bytes() of the same sizes (the factorization's
+ *   scratch followed by the attention's); contents undefined on return.
+ */
+size_t solar_fused_workspace_bytes(int B, int M, int N, int d, int r, solar_dtype_t dt);
+
+solar_status_t solar_svd_attention_fused(int B, int M, int N, int d, int r, solar_dtype_t dt,
+                                         const void* H, const void* C,
+                                         const void* Wq, const void* Wk, const void* Wv,
+                                         float scale, unsigned flags, float* S, float* V, void* O,
+                                         int* info, void* workspace, size_t workspace_bytes,
+                                         void* stream);
 
 /* ------------------------------------------------------------------------- *
  * Stage-level entry points.  The two calls above are exactly

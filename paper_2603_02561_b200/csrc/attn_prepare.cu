@@ -9,9 +9,8 @@
 // to 64 token slots.
 //
 // Two CTAs per user: one computes Key_r^T and T (W_K, W_Q), the other Value_r (W_V).
-// Each weight matrix is staged once in shared memory with coalesced 16-byte loads, all at
-// the start of the CTA; the small products then run out of shared memory with 4 outputs
-// per thread.
+// Each weight matrix is staged once in shared memory with coalesced 16-byte loads; the small
+// products then run out of shared memory with 4 outputs per thread.
 #include "solar_internal.cuh"
 
 namespace solar {
@@ -51,9 +50,12 @@ attn_prepare_kernel(const float* __restrict__ S, const float* __restrict__ V,
   __nv_bfloat16* Vpk = reinterpret_cast<__nv_bfloat16*>(wsb + lay.vpk_off);
   const __nv_bfloat16 zero = __float2bfloat16_rn(0.f);
 
+  // S and V come from the eigensolver, the weights from the caller (a kernel earlier on the
+  // stream may have written them), and the workspace may still be in use: nothing is read or
+  // written before the previous kernel has completed
+  pdl_wait();
   stage_weight<T, D>(role == 0 ? Wk : Wv, Ws, tid);
   if (role == 0) stage_weight<T, D>(Wq, Wq_s, tid);
-  pdl_wait();          // S and V come from the eigensolver; the workspace may still be in use before this
   for (int e = tid; e < D * rp; e += kPrepThreads) {
     const int k = e / rp, i = e % rp;
     VS[e] = i < r ? V[((size_t)b * D + k) * r + i] * (S != nullptr ? S[(size_t)b * r + i] : 1.f) : 0.f;

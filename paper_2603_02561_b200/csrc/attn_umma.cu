@@ -53,7 +53,7 @@ template <int D>
 __global__ void __launch_bounds__(128)
 attn_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmO,
                  const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUtensorMap tmV,
-                 int r, unsigned flags, __nv_bfloat16* __restrict__ O, int M) {
+                 int r, unsigned flags, __nv_bfloat16* __restrict__ O, int M, int early_c) {
   using Cfg = AttnCfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -86,9 +86,13 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
 
   if (tid == 0) {
     ptx::mbar_arrive_expect_tx(&bar_load, Cfg::C_BYTES + Cfg::t_bytes(np) + Cfg::V_BYTES);
+    // The packed operands come from the kernel before this one.  The candidate tile is the
+    // caller's: it may be fetched ahead of the wait only when an earlier kernel of the same
+    // library call has already waited for whatever ran before the call (early_c).
+    if (!early_c) pdl_wait();
 #pragma unroll
     for (int x = 0; x < Cfg::KB; ++x) ptx::tma_load_3d(sC + x * kBoxBytes, &tmC, &bar_load, x * 64, m0, b);
-    pdl_wait();        // the candidate tile is on its way; the packed operands come from the prepare kernel
+    if (early_c) pdl_wait();
 #pragma unroll
     for (int x = 0; x < Cfg::KB; ++x) {
 #pragma unroll
@@ -245,7 +249,7 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
 
 template <int D>
 cudaError_t launch_d(int B, int M, int r, const void* C, unsigned flags, void* O, const char* ws,
-                     const AttnWs& lay, cudaStream_t st) {
+                     const AttnWs& lay, bool early_c, cudaStream_t st) {
   using Cfg = AttnCfg<D>;
   CUtensorMap tmC, tmO, tmT, tmV;
   const uint64_t pu = lay.per_user;
@@ -262,7 +266,7 @@ cudaError_t launch_d(int B, int M, int r, const void* C, unsigned flags, void* O
   if (e != cudaSuccess) return e;
   const dim3 grid((M + kRows - 1) / kRows, B), block(128);
   return launch_pdl(attn_umma_kernel<D>, grid, block, Cfg::smem(np), st, tmC, tmO, tmT, tmV, r, flags,
-                    static_cast<__nv_bfloat16*>(O), M);
+                    static_cast<__nv_bfloat16*>(O), M, early_c ? 1 : 0);
 }
 
 }  // namespace
@@ -270,9 +274,9 @@ cudaError_t launch_d(int B, int M, int r, const void* C, unsigned flags, void* O
 bool attn_umma_supported(int d, solar_dtype_t dt) { return dt == SOLAR_BF16 && (d == 64 || d == 128); }
 
 cudaError_t launch_attn_umma(int B, int M, int d, int r, const void* C, unsigned flags, void* O,
-                             const char* ws, const AttnWs& lay, cudaStream_t st) {
-  return d == 64 ? launch_d<64>(B, M, r, C, flags, O, ws, lay, st)
-                 : launch_d<128>(B, M, r, C, flags, O, ws, lay, st);
+                             const char* ws, const AttnWs& lay, bool early_c, cudaStream_t st) {
+  return d == 64 ? launch_d<64>(B, M, r, C, flags, O, ws, lay, early_c, st)
+                 : launch_d<128>(B, M, r, C, flags, O, ws, lay, early_c, st);
 }
 
 }  // namespace solar

@@ -647,7 +647,7 @@ cudaError_t launch_eig(int B, int d, int r, solar_dtype_t dt, int route, int swe
   // AUTO and TRIDIAG: the tridiagonal route (with the Jacobi solve behind it in AUTO)
   if (route == SOLAR_ROUTE_AUTO || route == SOLAR_ROUTE_TRIDIAG)
     return launch_eig_tridiag(B, d, r, dt, route, sweep_cap, gpart, gram_status, splits, gsum, S, V, info,
-                              route_taken, st);
+                              route_taken, nullptr, st);
   EigTol tol;
   if (dt == SOLAR_BF16) {
     tol.eps_vec = 1e-3f; tol.floor_rel = 256.f * kUnit; tol.sweep_stop = 1e-3f;

@@ -77,7 +77,9 @@ template <int D, int RP> struct TriSmem {
   static constexpr int KT = SG + RP;                             // [RP] twist index (int)
   static constexpr int PART = KT + RP;                           // [2][NW][RP] per-warp partial results
   static constexpr int TRI_FLOATS = PART + 2 * C::NW * RP;
-  static constexpr int FLOATS = TRI_FLOATS > full_jacobi_floats<D>() ? TRI_FLOATS : full_jacobi_floats<D>();
+  static constexpr int EPI_FLOATS = 2 * D * RP + 2 * D * D;      // the projection epilogue: V Sigma, Key_r^T, two weights
+  static constexpr int M1 = TRI_FLOATS > full_jacobi_floats<D>() ? TRI_FLOATS : full_jacobi_floats<D>();
+  static constexpr int FLOATS = M1 > EPI_FLOATS ? M1 : EPI_FLOATS;
   static constexpr size_t BYTES = (size_t)FLOATS * sizeof(float);
   static_assert(DG % 4 == 0 && EO % 4 == 0 && E2 % 4 == 0 && XP % 4 == 0 && TP % 4 == 0 && PV % 4 == 0 &&
                 EM % 4 == 0 && WORK % 4 == 0 && VS % 4 == 0, "16-byte alignment of the regions");
@@ -279,12 +281,15 @@ struct TriTol {
   float sweep_stop;  // of the Jacobi fallback
 };
 
+// The eigensolve of user blockIdx.x; every thread of the CTA calls it and all leave together.
+// With want_vs, a certified tridiagonal result also leaves V Sigma at the start of the dynamic
+// shared memory ([D][rp], rp = r rounded up to 4, zero in the padding) and true is returned.
 template <int D, int RP>
-__global__ void __launch_bounds__(TriCfg<D>::NT, 1)
-eig_tridiag_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status, int splits,
-                   float* __restrict__ gsum, int r, int route, int sweep_cap, TriTol tol,
-                   float* __restrict__ S, float* __restrict__ V, int* __restrict__ info,
-                   int* __restrict__ route_taken) {
+__device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const int* __restrict__ gram_status,
+                                         int splits, float* __restrict__ gsum, int r, int route, int sweep_cap,
+                                         const TriTol& tol, bool want_vs, float* __restrict__ S,
+                                         float* __restrict__ V, int* __restrict__ info,
+                                         int* __restrict__ route_taken) {
   using Cfg = TriCfg<D>;
   using L = TriSmem<D, RP>;
   constexpr int NT = Cfg::NT, NW = Cfg::NW, RPT = Cfg::RPT, CPT = Cfg::CPT, NG = Cfg::NG, LD = Cfg::LD;
@@ -368,7 +373,7 @@ eig_tridiag_kernel(const float* __restrict__ gpart, const int* __restrict__ gram
       for (int e = tid; e < r; e += NT) S[(size_t)b * r + e] = qnan;
       if (tid == 0 && info) info[b] = lost ? SOLAR_INFO_DEVICE_WAIT : SOLAR_INFO_NONFINITE;
       if (tid == 0 && route_taken) route_taken[b] = 0;
-      return;
+      return false;
     }
   }
   if (tid < 32) {
@@ -710,7 +715,7 @@ eig_tridiag_kernel(const float* __restrict__ gpart, const int* __restrict__ gram
       __syncthreads();
       const float em = s_emax;
       if (em <= tol.ortho) break;                       // orthonormal to rounding
-      if (passes == 3 || !(em <= 0.25f)) { ok = false; if (tid == 0) s_why |= kWhyOrtho; break; }
+      if (passes == 6 || !(em <= 0.5f)) { ok = false; if (tid == 0) s_why |= kWhyOrtho; break; }
       ++passes;
       // rows i of V' for this warp: D / NW of them; lane = column(s)
       float ecol[NE][RP];
@@ -833,18 +838,28 @@ eig_tridiag_kernel(const float* __restrict__ gpart, const int* __restrict__ gram
           if (fabsf(v) > best) { best = fabsf(v); lead = v; }   // strict: lowest index wins a tie
         }
         sgn[tid] = lead < 0.f ? -1.f : 1.f;
-        if (tid < r) S[(size_t)b * r + tid] = sqrtf(fmaxf(m, 0.f) / sc);
+        const float sv = sqrtf(fmaxf(m, 0.f) / sc);
+        rho2[tid] = sv;
+        if (tid < r) S[(size_t)b * r + tid] = sv;
       }
       __syncthreads();
       for (int e = tid; e < D * r; e += NT) {
         const int i = e / r, j = e % r;
         V[(size_t)b * D * r + e] = Vc[i * RP + j] * sgn[j];
       }
+      if (want_vs) {
+        const int rp = (r + 3) & ~3;
+        float* vsig = smem;                            // over G: the residuals are done
+        for (int e = tid; e < D * rp; e += NT) {
+          const int i = e / rp, j = e % rp;
+          vsig[e] = j < r ? (Vc[i * RP + j] * sgn[j]) * rho2[j] : 0.f;
+        }
+      }
       if (tid == 0) {
         if (info) info[b] = ok ? 0 : SOLAR_INFO_NOT_CERTIFIED;
         if (route_taken) route_taken[b] = kRouteTridiag | (passes << 16) | (s_why << 24);
       }
-      return;
+      return want_vs;
     }
     __syncthreads();
   }
@@ -859,12 +874,258 @@ eig_tridiag_kernel(const float* __restrict__ gpart, const int* __restrict__ gram
   const float thr_abs2 = (kTolAbs * gmax * sc) * (kTolAbs * gmax * sc);
   full_jacobi_route<D, NT>(smem, s_flags, b, tid, r, sc, thr_abs2, tol.sweep_stop * tol.sweep_stop, s_why,
                            sweep_cap, S, V, info, route_taken);
+  return false;
+}
+
+// ---- optional epilogue: the factor-token projections of Eq. 11 for this user ---------------
+// Key_r = (V Sigma)^T W_K, Value_r = (V Sigma)^T W_V and the folded score operand
+// T = scale * W_Q Key_r^T, written to the attention workspace in the layout and with the
+// summation order of the stand-alone projection kernel, so that a forward pass which ends its
+// eigensolver CTAs with this epilogue needs one launch less and gives the same bits.
+struct FuseArgs {
+  const void* Wq; const void* Wk; const void* Wv;
+  float scale;
+  char* ws;            // attention workspace (all users)
+  AttnWs lay;
+  int mode;            // 0: no epilogue; 1: weights are bf16; 2: weights are fp32
+  int write_f32;       // also write the fp32 copies T and Value_r (read by the FFMA attention kernel)
+};
+
+// Stages W[D][D] (bf16 or fp32 in global memory) as fp32 in shared memory, as it is or
+// transposed.  All loads of a thread are issued before the first store.
+template <int D, int NT, bool TRANSPOSE>
+__device__ __forceinline__ void stage_weight_any(const void* __restrict__ W, int mode, float* __restrict__ Ws,
+                                                 int tid) {
+  constexpr int NV = D * D / 8 / NT;              // 8-element pieces per thread
+  static_assert(NV * NT * 8 == D * D, "whole pieces");
+  float x[NV][8];
+  if (mode == 1) {
+    const uint4* w = static_cast<const uint4*>(W);
+    uint4 raw[NV];
+#pragma unroll
+    for (int n = 0; n < NV; ++n) raw[n] = __ldg(w + tid + n * NT);
+#pragma unroll
+    for (int n = 0; n < NV; ++n) {
+      const uint32_t u[4] = {raw[n].x, raw[n].y, raw[n].z, raw[n].w};
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        x[n][2 * q] = __uint_as_float(u[q] << 16);
+        x[n][2 * q + 1] = __uint_as_float(u[q] & 0xffff0000u);
+      }
+    }
+  } else {
+    const float4* w = static_cast<const float4*>(W);
+#pragma unroll
+    for (int n = 0; n < NV; ++n) {
+      const float4 lo = __ldg(w + 2 * (tid + n * NT)), hi = __ldg(w + 2 * (tid + n * NT) + 1);
+      x[n][0] = lo.x; x[n][1] = lo.y; x[n][2] = lo.z; x[n][3] = lo.w;
+      x[n][4] = hi.x; x[n][5] = hi.y; x[n][6] = hi.z; x[n][7] = hi.w;
+    }
+  }
+#pragma unroll
+  for (int n = 0; n < NV; ++n) {
+    const int e0 = (tid + n * NT) * 8;            // element e0 = row * D + col
+    if (!TRANSPOSE) {
+      *reinterpret_cast<float4*>(Ws + e0) = make_float4(x[n][0], x[n][1], x[n][2], x[n][3]);
+      *reinterpret_cast<float4*>(Ws + e0 + 4) = make_float4(x[n][4], x[n][5], x[n][6], x[n][7]);
+    } else {
+      const int row = e0 / D, col = e0 % D;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) Ws[(col + u) * D + row] = x[n][u];
+    }
+  }
+}
+
+// 16-byte pieces of a packed bf16 operand row: eight fp32 values as their high halves (h = 0)
+// or as what the high halves leave over (h = 1).
+__device__ __forceinline__ uint4 pack8_bf16(const float (&x)[8], int h) {
+  uint32_t w[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    float a = x[2 * q], c = x[2 * q + 1];
+    if (h) {
+      a -= __bfloat162float(__float2bfloat16_rn(a));
+      c -= __bfloat162float(__float2bfloat16_rn(c));
+    }
+    const __nv_bfloat162 v = __floats2bfloat162_rn(a, c);
+    w[q] = *reinterpret_cast<const uint32_t*>(&v);
+  }
+  return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// vs_ready: V Sigma of this user already lies at sm[0 .. D * rp) (pitch rp = r rounded up to 4,
+// zero in the padding), left there by the eigensolver; otherwise it is read back from S and V.
+template <int D, int NT>
+__device__ __forceinline__ void prepare_epilogue(float* __restrict__ sm, int b, int r, const float* __restrict__ S,
+                                                 const float* __restrict__ V, const FuseArgs& fa, bool vs_ready,
+                                                 int tid) {
+  const int rp = (r + 3) & ~3;          // token pitch: rows of VS / KrT are read 4 at a time
+  float* VS = sm;                       // [D][rp]  V Sigma (zero in the padding)
+  float* KrT = VS + D * rp;             // [D][rp]  Key_r^T; later Value_r^T
+  float* W0 = KrT + D * rp;             // [D][D]   W_K, then W_V
+  float* W1 = W0 + D * D;               // [D][D]   W_Q^T; later T^T [r][D]
+  char* wsb = fa.ws + (size_t)b * fa.lay.per_user;
+  float* Tf = reinterpret_cast<float*>(wsb + fa.lay.tf_off);
+  float* Vr = reinterpret_cast<float*>(wsb + fa.lay.vr_off);
+  __nv_bfloat16* Tpk = reinterpret_cast<__nv_bfloat16*>(wsb + fa.lay.tpk_off);
+  __nv_bfloat16* Vpk = reinterpret_cast<__nv_bfloat16*>(wsb + fa.lay.vpk_off);
+  const int nt4 = rp / 4;               // groups of four tokens
+  const int ntile = nt4 * (D / 4);      // 4 x 4 output tiles of each of the three products
+  constexpr int MAXT = 2;               // tiles per thread (kept in registers across a barrier)
+  const uint4 z4 = make_uint4(0u, 0u, 0u, 0u);
+
+  stage_weight_any<D, NT, false>(fa.Wk, fa.mode, W0, tid);
+  stage_weight_any<D, NT, true>(fa.Wq, fa.mode, W1, tid);
+  if (!vs_ready)
+    for (int e = tid; e < D * rp; e += NT) {
+      const int k = e / rp, i = e % rp;
+      VS[e] = i < r ? V[((size_t)b * D + k) * r + i] * S[(size_t)b * r + i] : 0.f;
+    }
+  // Zero padding of the packed operands, 16 bytes at a time.  The tensor-core attention kernel
+  // multiplies over np = 16 ceil(r / 16) token slots only (slots r .. r8-1, r8 = r rounded up to
+  // 8, are written as zeros with the data below); the FFMA kernels' callers want all 64.
+  const int r8 = (r + 7) & ~7;
+  const int pad_to = fa.write_f32 ? kTokenSlots : ((r + 15) & ~15);
+  for (int e = tid; e < 2 * (pad_to - r8) * (D / 8); e += NT) {
+    const int h = e / ((pad_to - r8) * (D / 8)), rem = e % ((pad_to - r8) * (D / 8));
+    reinterpret_cast<uint4*>(Tpk + ((size_t)h * kTokenSlots + r8) * D)[rem] = z4;
+  }
+  for (int e = tid; e < 2 * D * ((pad_to - r8) / 8); e += NT) {
+    const int row = e / ((pad_to - r8) / 8), c = e % ((pad_to - r8) / 8);
+    reinterpret_cast<uint4*>(Vpk + (size_t)row * kTokenSlots + r8)[c] = z4;      // row runs over [2][D]
+  }
+  __syncthreads();
+  // acc[a][c] = sum_k VS[k][i0 + a] W0[k][j0 + c]: a 4 x 4 tile per thread, two 16-byte reads per
+  // 16 FMAs, every output summed over k in ascending order
+  auto project = [&](float (&acc)[4][4], int i0, int j0) {
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) acc[a][c] = 0.f;
+#pragma unroll 4
+    for (int k = 0; k < D; ++k) {
+      const float4 w = *reinterpret_cast<const float4*>(W0 + k * D + j0);
+      const float4 v = *reinterpret_cast<const float4*>(VS + k * rp + i0);
+      const float ww[4] = {w.x, w.y, w.z, w.w}, vv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[a][c] = fmaf(vv[a], ww[c], acc[a][c]);
+    }
+  };
+  // Key_r^T [j][i]
+  for (int t = tid; t < ntile; t += NT) {
+    const int j0 = (t % (D / 4)) * 4, i0 = (t / (D / 4)) * 4;
+    float acc[4][4];
+    project(acc, i0, j0);
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+      *reinterpret_cast<float4*>(KrT + (j0 + c) * rp + i0) = make_float4(acc[0][c], acc[1][c], acc[2][c], acc[3][c]);
+  }
+  __syncthreads();
+  // T[k][i] = scale * sum_j Wq[k][j] Key_r[i][j]: tile of four rows k and four tokens i; kept in
+  // registers until W_Q is done with, then laid down over it as T^T [i][D] (the packed rows)
+  float tacc[MAXT][4][4];
+#pragma unroll
+  for (int n = 0; n < MAXT; ++n) {
+    const int t = tid + n * NT;
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tacc[n][a][c] = 0.f;
+    if (t < ntile) {
+      const int i0 = (t % nt4) * 4, k0 = (t / nt4) * 4;
+#pragma unroll 4
+      for (int j = 0; j < D; ++j) {
+        const float4 w = *reinterpret_cast<const float4*>(W1 + j * D + k0);      // W_Q[k0 ..][j]
+        const float4 kr = *reinterpret_cast<const float4*>(KrT + j * rp + i0);
+        const float ww[4] = {w.x, w.y, w.z, w.w}, kk[4] = {kr.x, kr.y, kr.z, kr.w};
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+          for (int c = 0; c < 4; ++c) tacc[n][a][c] = fmaf(ww[a], kk[c], tacc[n][a][c]);
+      }
+    }
+  }
+  __syncthreads();
+  stage_weight_any<D, NT, false>(fa.Wv, fa.mode, W0, tid);       // W_K is done with
+#pragma unroll
+  for (int n = 0; n < MAXT; ++n) {
+    const int t = tid + n * NT;
+    if (t < ntile) {
+      const int i0 = (t % nt4) * 4, k0 = (t / nt4) * 4;
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+        *reinterpret_cast<float4*>(W1 + (i0 + c) * D + k0) =
+            make_float4(tacc[n][0][c] * fa.scale, tacc[n][1][c] * fa.scale, tacc[n][2][c] * fa.scale,
+                        tacc[n][3][c] * fa.scale);
+    }
+  }
+  __syncthreads();
+  // T^T out: 16-byte pieces of the packed rows (tokens r .. r8-1 are zero rows), and the fp32 copy
+  for (int e = tid; e < 2 * r8 * (D / 8); e += NT) {
+    const int h = e / (r8 * (D / 8)), rem = e % (r8 * (D / 8)), i = rem / (D / 8), c = rem % (D / 8);
+    const float4 lo = *reinterpret_cast<const float4*>(W1 + i * D + 8 * c);
+    const float4 hi = *reinterpret_cast<const float4*>(W1 + i * D + 8 * c + 4);
+    float x[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+    if (i >= r) {
+#pragma unroll
+      for (int u = 0; u < 8; ++u) x[u] = 0.f;
+    }
+    reinterpret_cast<uint4*>(Tpk + ((size_t)h * kTokenSlots + i) * D)[c] = pack8_bf16(x, h);
+  }
+  if (fa.write_f32)
+    for (int e = tid; e < D * r; e += NT) Tf[e] = W1[(e % r) * D + e / r];
+  // Value_r, kept in registers until Key_r^T is done with, then laid down over it as
+  // Value_r^T [j][rp] (the packed operand's rows)
+#pragma unroll
+  for (int n = 0; n < MAXT; ++n) {
+    const int t = tid + n * NT;
+    if (t < ntile) project(tacc[n], (t / (D / 4)) * 4, (t % (D / 4)) * 4);
+  }
+  __syncthreads();
+#pragma unroll
+  for (int n = 0; n < MAXT; ++n) {
+    const int t = tid + n * NT;
+    if (t < ntile) {
+      const int j0 = (t % (D / 4)) * 4, i0 = (t / (D / 4)) * 4;
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+        *reinterpret_cast<float4*>(KrT + (j0 + c) * rp + i0) =
+            make_float4(tacc[n][0][c], tacc[n][1][c], tacc[n][2][c], tacc[n][3][c]);
+    }
+  }
+  __syncthreads();
+  for (int e = tid; e < 2 * D * (r8 / 8); e += NT) {
+    const int h = e / (D * (r8 / 8)), rem = e % (D * (r8 / 8)), j = rem / (r8 / 8), c = rem % (r8 / 8);
+    float x[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) x[u] = (8 * c + u < r) ? KrT[j * rp + 8 * c + u] : 0.f;
+    reinterpret_cast<uint4*>(Vpk + ((size_t)h * D + j) * kTokenSlots)[c] = pack8_bf16(x, h);
+  }
+  if (fa.write_f32)
+    for (int e = tid; e < r * D; e += NT) Vr[e] = KrT[(e % D) * rp + e / D];
+}
+
+template <int D, int RP>
+__global__ void __launch_bounds__(TriCfg<D>::NT, 1)
+eig_tridiag_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status, int splits,
+                   float* __restrict__ gsum, int r, int route, int sweep_cap, TriTol tol,
+                   float* __restrict__ S, float* __restrict__ V, int* __restrict__ info,
+                   int* __restrict__ route_taken, FuseArgs fa) {
+  const bool vs_ready = eig_user<D, RP>(gpart, gram_status, splits, gsum, r, route, sweep_cap, tol, fa.mode != 0, S, V,
+                                        info, route_taken);
+  if (fa.mode != 0) {
+    extern __shared__ __align__(16) float smem[];
+    __syncthreads();                    // S and V of this user are written (and visible to the CTA)
+    prepare_epilogue<D, TriCfg<D>::NT>(smem, blockIdx.x, r, S, V, fa, vs_ready, threadIdx.x);
+  }
 }
 
 template <int D, int RP>
 cudaError_t launch_tri(int B, int r, int route, int sweep_cap, TriTol tol, const float* gpart,
                        const int* gram_status, int splits, float* gsum, float* S, float* V, int* info,
-                       int* route_taken, cudaStream_t st) {
+                       int* route_taken, const FuseArgs& fa, cudaStream_t st) {
   using L = TriSmem<D, RP>;
   static bool attr_set[64] = {};
   int dev = 0;
@@ -877,14 +1138,22 @@ cudaError_t launch_tri(int B, int r, int route, int sweep_cap, TriTol tol, const
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
   return launch_pdl(eig_tridiag_kernel<D, RP>, dim3(B), dim3(TriCfg<D>::NT), L::BYTES, st, gpart, gram_status,
-                    splits, gsum, r, route, sweep_cap, tol, S, V, info, route_taken);
+                    splits, gsum, r, route, sweep_cap, tol, S, V, info, route_taken, fa);
 }
 
 }  // namespace
 
 cudaError_t launch_eig_tridiag(int B, int d, int r, solar_dtype_t dt, int route, int sweep_cap,
                                const float* gpart, const int* gram_status, int splits, float* gsum,
-                               float* S, float* V, int* info, int* route_taken, cudaStream_t st) {
+                               float* S, float* V, int* info, int* route_taken, const EigFuse* fuse,
+                               cudaStream_t st) {
+  FuseArgs fa = {};
+  if (fuse != nullptr) {
+    fa.Wq = fuse->Wq; fa.Wk = fuse->Wk; fa.Wv = fuse->Wv; fa.scale = fuse->scale;
+    fa.ws = fuse->attn_ws; fa.lay = attn_ws_layout(d, r);
+    fa.mode = (dt == SOLAR_BF16) ? 1 : 2;
+    fa.write_f32 = !attn_umma_supported(d, dt);
+  }
   TriTol tol;
   if (dt == SOLAR_BF16) {
     tol.eps_vec = 1e-3f; tol.floor_rel = 64.f * kUnit; tol.ortho = 4e-6f; tol.sweep_stop = 1e-3f;
@@ -894,13 +1163,13 @@ cudaError_t launch_eig_tridiag(int B, int d, int r, solar_dtype_t dt, int route,
   const bool wide = r > 32;
   switch (d) {
     case 32:
-      return launch_tri<32, 32>(B, r, route, sweep_cap, tol, gpart, gram_status, splits, gsum, S, V, info, route_taken, st);
+      return launch_tri<32, 32>(B, r, route, sweep_cap, tol, gpart, gram_status, splits, gsum, S, V, info, route_taken, fa, st);
     case 64:
-      return wide ? launch_tri<64, 64>(B, r, route, sweep_cap, tol, gpart, gram_status, splits, gsum, S, V, info, route_taken, st)
-                  : launch_tri<64, 32>(B, r, route, sweep_cap, tol, gpart, gram_status, splits, gsum, S, V, info, route_taken, st);
+      return wide ? launch_tri<64, 64>(B, r, route, sweep_cap, tol, gpart, gram_status, splits, gsum, S, V, info, route_taken, fa, st)
+                  : launch_tri<64, 32>(B, r, route, sweep_cap, tol, gpart, gram_status, splits, gsum, S, V, info, route_taken, fa, st);
     case 128:
-      return wide ? launch_tri<128, 64>(B, r, route, sweep_cap, tol, gpart, gram_status, splits, gsum, S, V, info, route_taken, st)
-                  : launch_tri<128, 32>(B, r, route, sweep_cap, tol, gpart, gram_status, splits, gsum, S, V, info, route_taken, st);
+      return wide ? launch_tri<128, 64>(B, r, route, sweep_cap, tol, gpart, gram_status, splits, gsum, S, V, info, route_taken, fa, st)
+                  : launch_tri<128, 32>(B, r, route, sweep_cap, tol, gpart, gram_status, splits, gsum, S, V, info, route_taken, fa, st);
     default: return cudaErrorInvalidValue;
   }
 }

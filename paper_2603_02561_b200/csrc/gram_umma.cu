@@ -65,6 +65,9 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tmap, float* __restrict__ g
 
   if (warp == 0 && lane == 0) {
     // ---- producer: one TMA tile per stage ------------------------------------------
+    // H is the caller's: whatever wrote it earlier on the stream must have completed before the
+    // first tile is fetched (the set-up above did overlap that kernel's tail)
+    pdl_wait();
     int issued = 0;
     for (int t = 0; t < ntiles; ++t) {
       const int st = t % STAGES;
@@ -108,8 +111,8 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tmap, float* __restrict__ g
   __syncwarp();
   ptx::tc_fence_after_sync();
   float* out = gpart + ((size_t)b * splits + s) * D * D;
-  // H has been streamed without waiting for the previous kernel on the stream (it may
-  // still be reading this workspace); nothing is written before it has completed.
+  // nothing is written before the previous kernel on the stream (it may still be reading this
+  // workspace) has completed
   pdl_wait();
   if (done && *err == 0) {
     // M = 128: accumulator row i sits in lane i.  M = 64: rows 16q .. 16q+15 sit in lanes

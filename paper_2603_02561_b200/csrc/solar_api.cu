@@ -34,6 +34,19 @@ solar_status_t check_ws(const void* ws, size_t have, size_t need) {
 
 solar_status_t from_cuda(cudaError_t e) { return e == cudaSuccess ? SOLAR_OK : SOLAR_ERR_CUDA; }
 
+// Scores, softmax, weighted sum from a prepared workspace.  early_c: an earlier kernel of the
+// same library call has already waited for whatever ran before the call, so the candidate tile
+// may be fetched ahead of this kernel's own wait.
+solar_status_t attn_apply_impl(int B, int M, int d, int r, solar_dtype_t dt, const void* C, unsigned flags,
+                               void* O, const char* ws, bool early_c, cudaStream_t st) {
+  if (attn_umma_supported(d, dt))
+    return from_cuda(launch_attn_umma(B, M, d, r, C, flags, O, ws, attn_ws_layout(d, r), early_c, st));
+  return from_cuda(launch_attn_simt(B, M, d, r, dt, C, flags, O, ws, attn_ws_layout(d, r), st));
+}
+
+// Workspace of the fused forward call: the factorization's, then the attention's.
+size_t fused_attn_offset(int B, int N, int d) { return align_up(factor_ws_bytes(B, N, d), 256); }
+
 }  // namespace
 
 extern "C" {
@@ -158,12 +171,8 @@ solar_status_t solar_attn_apply(int B, int M, int d, int r, solar_dtype_t dt, co
   SOLAR_TRY(check_ptr(C));
   SOLAR_TRY(check_ptr(O));
   SOLAR_TRY(check_ws(workspace, workspace_bytes, attn_ws_bytes(B, d, r)));
-  const cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (attn_umma_supported(d, dt))
-    return from_cuda(launch_attn_umma(B, M, d, r, C, flags, O, static_cast<const char*>(workspace),
-                                      attn_ws_layout(d, r), st));
-  return from_cuda(launch_attn_simt(B, M, d, r, dt, C, flags, O, static_cast<const char*>(workspace),
-                                    attn_ws_layout(d, r), st));
+  return attn_apply_impl(B, M, d, r, dt, C, flags, O, static_cast<const char*>(workspace), false,
+                         static_cast<cudaStream_t>(stream));
 }
 
 solar_status_t solar_svd_attention_fwd(int B, int M, int N, int d, int r, solar_dtype_t dt,
@@ -185,7 +194,46 @@ solar_status_t solar_svd_attention_fwd(int B, int M, int N, int d, int r, solar_
   SOLAR_TRY(check_ws(workspace, workspace_bytes, attn_ws_bytes(B, d, r)));
   SOLAR_TRY(solar_attn_prepare(B, d, r, dt, S, V, Wq, Wk, Wv, scale, workspace, workspace_bytes,
                                stream));
-  return solar_attn_apply(B, M, d, r, dt, C, flags, O, workspace, workspace_bytes, stream);
+  return attn_apply_impl(B, M, d, r, dt, C, flags, O, static_cast<const char*>(workspace), true,
+                         static_cast<cudaStream_t>(stream));
+}
+
+size_t solar_fused_workspace_bytes(int B, int M, int N, int d, int r, solar_dtype_t dt) {
+  if (check_dims(B, M, N, d, r, dt) != SOLAR_OK) return 0;
+  return fused_attn_offset(B, N, d) + align_up(attn_ws_bytes(B, d, r), 256);
+}
+
+solar_status_t solar_svd_attention_fused(int B, int M, int N, int d, int r, solar_dtype_t dt,
+                                         const void* H, const void* C, const void* Wq, const void* Wk,
+                                         const void* Wv, float scale, unsigned flags, float* S, float* V,
+                                         void* O, int* info, void* workspace, size_t workspace_bytes,
+                                         void* stream) {
+  SOLAR_TRY(check_dims(B, M, N, d, r, dt));
+  if (flags & ~(unsigned)SOLAR_FLAG_NO_SOFTMAX) return SOLAR_ERR_UNSUPPORTED;
+  if (B == 0) return SOLAR_OK;
+  SOLAR_TRY(check_ptr(H));
+  SOLAR_TRY(check_ptr(S));
+  SOLAR_TRY(check_ptr(V));
+  SOLAR_TRY(check_ptr(Wq));
+  SOLAR_TRY(check_ptr(Wk));
+  SOLAR_TRY(check_ptr(Wv));
+  if (M > 0) { SOLAR_TRY(check_ptr(C)); SOLAR_TRY(check_ptr(O)); }
+  if (info != nullptr && (reinterpret_cast<uintptr_t>(info) & 3u)) return SOLAR_ERR_INVALID_ARG;
+  SOLAR_TRY(check_ws(workspace, workspace_bytes, solar_fused_workspace_bytes(B, M, N, d, r, dt)));
+  const cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* ws = static_cast<char*>(workspace);
+  char* attn_ws = ws + fused_attn_offset(B, N, d);
+  // streaming pass over H (the first kernel of the call: it waits for what ran before)
+  SOLAR_TRY(solar_gram_partials(B, N, d, dt, H, workspace, factor_ws_bytes(B, N, d), stream));
+  // eigensolve; every user's CTA ends with that user's factor-token projections
+  const GramPlan plan = gram_plan(B, N);
+  const int* status = reinterpret_cast<const int*>(ws + gram_status_offset(B, N, d));
+  float* gsum = reinterpret_cast<float*>(ws + gram_sum_offset(B, N, d));
+  const EigFuse fuse = {Wq, Wk, Wv, scale, attn_ws};
+  SOLAR_TRY(from_cuda(launch_eig_tridiag(B, d, r, dt, SOLAR_ROUTE_AUTO, kMaxSweeps, reinterpret_cast<const float*>(ws),
+                                         status, plan.splits, gsum, S, V, info, nullptr, &fuse, st)));
+  if (M == 0) return SOLAR_OK;
+  return attn_apply_impl(B, M, d, r, dt, C, flags, O, attn_ws, true, st);
 }
 
 size_t solar_backward_workspace_bytes(int B, int M, int N, int d, int r, solar_dtype_t dt) {

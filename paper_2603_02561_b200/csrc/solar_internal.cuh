@@ -149,9 +149,17 @@ cudaError_t launch_gram_umma(int B, int N, int d, const void* H, float* gpart, i
 cudaError_t launch_eig(int B, int d, int r, solar_dtype_t dt, int route, int sweep_cap, int force_iters,
                        const float* gpart, const int* gram_status, int splits, float* gsum, float* S,
                        float* V, int* info, int* route_taken, cudaStream_t st);
+// The eigensolver CTA of a user may end with that user's factor-token projections (Eq. 11):
+// weights in the storage type, the attention workspace of all users.
+struct EigFuse {
+  const void* Wq; const void* Wk; const void* Wv;
+  float scale;
+  char* attn_ws;
+};
 cudaError_t launch_eig_tridiag(int B, int d, int r, solar_dtype_t dt, int route, int sweep_cap,
                                const float* gpart, const int* gram_status, int splits, float* gsum,
-                               float* S, float* V, int* info, int* route_taken, cudaStream_t st);
+                               float* S, float* V, int* info, int* route_taken, const EigFuse* fuse,
+                               cudaStream_t st);
 int eig_subspace_dim(int d, int r);
 cudaError_t launch_project_us(int B, int N, int d, int r, solar_dtype_t dt, const void* H,
                               const float* V, void* US, cudaStream_t st);
@@ -180,7 +188,7 @@ cudaError_t launch_flash_factored(int B, int M, int N, int d, int r, const void*
                                   const char* ws, const AttnWs& lay, cudaStream_t st);
 bool attn_umma_supported(int d, solar_dtype_t dt);
 cudaError_t launch_attn_umma(int B, int M, int d, int r, const void* C, unsigned flags, void* O,
-                             const char* ws, const AttnWs& lay, cudaStream_t st);
+                             const char* ws, const AttnWs& lay, bool early_c, cudaStream_t st);
 
 // ---- programmatic dependent launch ---------------------------------------------------
 // The four kernels of a forward pass run back to back on one stream.  Launched with this

@@ -35,6 +35,9 @@ SIGNATURES = {
     "solar_lowrank_factor": (_c_int, [_c_int] * 5 + [_c_int] + [_c_vp] * 5 + [_c_vp, _c_size, _c_vp]),
     "solar_svd_attention_fwd": (_c_int, [_c_int] * 5 + [_c_int] + [_c_vp] * 6 +
                                 [_c_float, _c_uint, _c_vp, _c_vp, _c_size, _c_vp]),
+    "solar_fused_workspace_bytes": (_c_size, [_c_int] * 5 + [_c_int]),
+    "solar_svd_attention_fused": (_c_int, [_c_int] * 5 + [_c_int] + [_c_vp] * 5 + [_c_float, _c_uint] +
+                                  [_c_vp] * 4 + [_c_vp, _c_size, _c_vp]),
     "solar_gram_splits": (_c_int, [_c_int] * 3 + [_c_int]),
     "solar_gram_partials": (_c_int, [_c_int] * 3 + [_c_int, _c_vp, _c_vp, _c_size, _c_vp]),
     "solar_eig_from_partials": (_c_int, [_c_int] * 4 + [_c_int] + [_c_vp] * 3 + [_c_vp, _c_size, _c_vp]),
@@ -285,6 +288,38 @@ def attn_apply(C, r, flags, O, workspace, stream=None):
     _check(lib().solar_attn_apply(B, M, d, r, dtype_code(C.dtype), _ptr(C), int(flags), _ptr(O),
                                   _ptr(workspace), workspace.numel(), _stream(stream)),
            "solar_attn_apply")
+
+
+def fused_workspace_bytes(B, M, N, d, r, dtype) -> int:
+    return int(lib().solar_fused_workspace_bytes(B, M, N, d, r, dtype_code(dtype)))
+
+
+def alloc_fused_workspace(B, M, N, d, r, dtype, device="cuda") -> torch.Tensor:
+    return torch.empty(max(fused_workspace_bytes(B, M, N, d, r, dtype), 256), dtype=torch.uint8, device=device)
+
+
+def svd_attention_fused(H, C, Wq, Wk, Wv, r, scale, flags=0, S=None, V=None, O=None, info=None,
+                        workspace=None, stream=None):
+    """solar_svd_attention_fused: the whole forward pass (H, C, weights -> S, V, O) in one call."""
+    B, N, d = H.shape
+    M = C.shape[1]
+    _need(H, (B, N, d), H.dtype, "H"); _need(C, (B, M, d), H.dtype, "C")
+    for nm, W in (("Wq", Wq), ("Wk", Wk), ("Wv", Wv)):
+        _need(W, (d, d), H.dtype, nm)
+    dev = H.device
+    S = torch.empty(B, r, dtype=torch.float32, device=dev) if S is None else S
+    V = torch.empty(B, d, r, dtype=torch.float32, device=dev) if V is None else V
+    O = torch.empty_like(C) if O is None else O
+    _need(S, (B, r), torch.float32, "S"); _need(V, (B, d, r), torch.float32, "V"); _need(O, (B, M, d), H.dtype, "O")
+    if info is not None:
+        _need(info, (B,), torch.int32, "info")
+    if workspace is None:
+        workspace = alloc_fused_workspace(B, M, N, d, r, H.dtype, dev)
+    st = lib().solar_svd_attention_fused(B, M, N, d, r, dtype_code(H.dtype), _ptr(H), _ptr(C), _ptr(Wq), _ptr(Wk),
+                                         _ptr(Wv), float(scale), int(flags), _ptr(S), _ptr(V), _ptr(O), _ptr(info),
+                                         _ptr(workspace), workspace.numel(), _stream(stream))
+    _check(st, "solar_svd_attention_fused")
+    return O, S, V
 
 
 def forward(H, C, Wq, Wk, Wv, r, scale, flags=0, workspace=None, stream=None):
