@@ -7,7 +7,10 @@
 //        thread's registers; the probabilities go back to shared memory as bf16 high/low
 //   tcgen05.mma: O [128 x d] = P Value_r (hi*hi + hi*lo + lo*hi), fp32 in tensor memory
 //   tcgen05.ld -> bf16 -> shared memory -> TMA store (rows past M are clipped)
-// The M x r score matrix never leaves the SM.  Every wait is bounded; if one runs out the
+// The M x r score matrix never leaves the SM.  Shared and tensor memory are reused along the
+// way -- the candidate tile's buffer holds the probabilities once the scores are formed and
+// the output tile after that; the output accumulator takes the scores' columns -- so that five
+// CTAs (d = 64, r <= 32) share an SM and keep enough bytes in flight for the HBM.  Every wait is bounded; if one runs out the
 // tile's output rows are written as NaN.
 #include "sm100_ptx.cuh"
 #include "solar_internal.cuh"
@@ -19,7 +22,6 @@ namespace {
 constexpr int kRows = 128;                 // candidate rows per CTA = accumulator lanes
 constexpr int kBoxBytes = kRows * 128;     // one 64-column box of a 128-row tile
 constexpr int kErrLoad = 0x21, kErrScores = 0x22, kErrOut = 0x23;
-constexpr int kScoreCols = 64;             // tensor-memory columns reserved for the scores
 
 template <int D> struct AttnCfg {
   static constexpr int KB = D / 64;                               // 64-wide K boxes of the score GEMM
@@ -27,14 +29,25 @@ template <int D> struct AttnCfg {
   // T^T hi/lo: [2][KB][np rows][128 B], np = 16 * ceil(r / 16) token rows (known at launch)
   __host__ __device__ static constexpr int t_bytes(int np) { return 2 * KB * np * 128; }
   static constexpr int V_BYTES = 2 * D * 128;                     // Value_r^T hi/lo: [2][D rows][128 B]
-  static constexpr int P_BYTES = 2 * kBoxBytes;                   // probabilities hi/lo
-  static constexpr size_t smem(int np) { return (size_t)C_BYTES + t_bytes(np) + V_BYTES + P_BYTES + 1024; }
-  static constexpr int TMEM_COLS = (D == 64) ? 128 : 256;         // scores (64) + output (D), power of two
+  // Probabilities hi/lo: [2][128 rows][128 B], or [2][128 rows][64 B] (64-byte swizzle) when
+  // np <= 32.  They lie over the candidate tile when they fit there (always but d = 64, np > 32).
+  __host__ __device__ static constexpr bool p_narrow(int np) { return np <= 32; }
+  __host__ __device__ static constexpr int p_bytes(int np) { return p_narrow(np) ? kBoxBytes : 2 * kBoxBytes; }
+  __host__ __device__ static constexpr bool p_over_c(int np) { return p_bytes(np) <= C_BYTES; }
+  static constexpr size_t smem(int np) {
+    return (size_t)C_BYTES + t_bytes(np) + V_BYTES + (p_over_c(np) ? 0 : p_bytes(np)) + 1024;
+  }
+  static constexpr int TMEM_COLS = D;                             // scores (<= 64 columns), then the output (D)
 };
 
 // Byte offset of 16-byte chunk c of row `row` in a 128-byte-swizzled tile of 128-byte rows.
 __device__ __forceinline__ uint32_t swz(int row, int c) {
   return (uint32_t)row * 128u + (uint32_t)((c ^ (row & 7)) << 4);
+}
+// The same for a 64-byte-swizzled tile of 64-byte rows (4 chunks per row; address bits 4-5 are
+// XORed with bits 7-8, i.e. with row / 2).
+__device__ __forceinline__ uint32_t swz64(int row, int c) {
+  return (uint32_t)row * 64u + (uint32_t)((c ^ ((row >> 1) & 3)) << 4);
 }
 
 // 2^x by the special-function unit (2 ulp; the probabilities are rounded to bf16 pairs anyway).
@@ -68,7 +81,9 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
   const int np = (r + 15) & ~15;              // token slots the GEMMs run over (multiple of 16)
   const int t_tile = np * 128;                // bytes of one [np rows][128 B] tile of T^T
   uint8_t* sV = sT + Cfg::t_bytes(np);        // [2][D rows][128 B]   (a multiple of 2 KB further on)
-  uint8_t* sP = sV + Cfg::V_BYTES;            // [2][128 rows][128 B]
+  const bool p64 = Cfg::p_narrow(np);         // probabilities in 64-byte rows
+  uint8_t* sP = Cfg::p_over_c(np) ? sC : sV + Cfg::V_BYTES;   // [2][128 rows][128 or 64 B]
+  const int p_half = p64 ? kBoxBytes / 2 : kBoxBytes;          // bytes of one of the two halves
 
   if (tid == 0) {
     s_err = 0;
@@ -81,7 +96,7 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
   ptx::tc_fence_before_sync();
   __syncthreads();
   ptx::tc_fence_after_sync();
-  const uint32_t tmem_s = s_tmem, tmem_o = s_tmem + kScoreCols;
+  const uint32_t tmem_s = s_tmem, tmem_o = s_tmem;   // the output takes the scores' columns once they are read
   volatile int* err = &s_err;
 
   if (tid == 0) {
@@ -178,8 +193,9 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
         hi[q] = pack_bf16(h0, h1);
         lo[q] = pack_bf16(x0 - h0, x1 - h1);
       }
-      *reinterpret_cast<uint4*>(sP + swz(tid, c)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-      *reinterpret_cast<uint4*>(sP + kBoxBytes + swz(tid, c)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+      const uint32_t off = p64 ? swz64(tid, c) : swz(tid, c);
+      *reinterpret_cast<uint4*>(sP + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+      *reinterpret_cast<uint4*>(sP + p_half + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
     }
   }
   ptx::fence_proxy_async_smem();
@@ -194,11 +210,12 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
       bool acc = false;
 #pragma unroll
       for (int term = 0; term < 3; ++term) {
-        const uint32_t pa = ptx::smem_u32(sP) + (term == 2 ? kBoxBytes : 0);
+        const uint32_t pa = ptx::smem_u32(sP) + (term == 2 ? p_half : 0);
         const uint32_t vb = ptx::smem_u32(sV) + (term == 1 ? D * 128 : 0);
         for (int kk = 0; kk < np / 16; ++kk) {
-          ptx::umma_bf16_ss(tmem_o, ptx::umma_smem_desc(pa + kk * 32, 0, 1024),
-                            ptx::umma_smem_desc(vb + kk * 32, 0, 1024), idesc, acc);
+          const uint64_t ad = p64 ? ptx::umma_smem_desc_sw(pa + kk * 32, 0, 512, 4)     // 64-byte rows
+                                  : ptx::umma_smem_desc(pa + kk * 32, 0, 1024);
+          ptx::umma_bf16_ss(tmem_o, ad, ptx::umma_smem_desc(vb + kk * 32, 0, 1024), idesc, acc);
           acc = true;
         }
       }

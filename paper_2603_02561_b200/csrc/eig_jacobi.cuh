@@ -30,6 +30,7 @@ constexpr int kWhySweepCap = 8;     // the Ritz Jacobi hit its sweep cap
 constexpr int kWhyCholesky = 16;    // non-finite pivot in the Cholesky-QR
 constexpr int kWhyOrtho = 32;       // tridiagonal route: vectors of a cluster came out dependent
 constexpr int kWhyTrace = 64;       // tridiagonal route: trace of T differs from trace of G, or not finite
+constexpr int kWhyGap = 128;        // tridiagonal route: a gap between kept eigenvalues is too small for its accuracy
 
 // Rotation J = [[c, s], [-s, c]] that annihilates g_pq of the 2x2 symmetric block
 // [[a, g], [g, b]]; identity when g is negligible (or not a number).  Returned

@@ -22,9 +22,10 @@
 //      |gamma_k|): inverse iteration from the best unit vector, O(d) per vector, no pivoting.
 //   5. Back-transformation V = Q Z: four threads per vector, each applying the d-2 reflectors to
 //      its quarter of the rows held in registers.
-//   6. A first-order symmetric orthogonalisation V <- V (I - (V^T V - I)/2), repeated while
-//      V^T V - I is above the rounding level (vectors of close eigenvalues come out of step 4
-//      with a mutual error of order eps |T| / gap).
+//   6. Gram-Schmidt passes in matrix form, V <- V (I - strict_upper(V^T V - I)) D^-1, repeated
+//      while V^T V - I is above the rounding level (vectors of close eigenvalues come out of
+//      step 4 with a mutual error of order eps |T| / gap); a column is only ever corrected by
+//      the columns of larger eigenvalues.
 //   7. Rayleigh quotients theta_i = v_i^T G v_i and residuals G v_i - theta_i v_i against the
 //      ORIGINAL G: the result is accepted only if every residual is small against its gap (or
 //      at the rounding floor), V^T V = I to rounding, and trace(T) = trace(G); otherwise the
@@ -278,6 +279,7 @@ struct TriTol {
   float eps_vec;     // bound on sin(angle) of a kept vector implied by its residual and gap
   float floor_rel;   // residuals below floor_rel * theta_1 are at the rounding level of fp32
   float ortho;       // largest |V^T V - I| entry that needs no further orthogonalisation
+  float gap_min;     // smallest gap between kept eigenvalues, relative to the largest, the route is trusted with
   float sweep_stop;  // of the Jacobi fallback
 };
 
@@ -491,7 +493,23 @@ __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const 
       lam = 0.5f * (lo + hi);
       if (wg == 0) lamv[j] = lam;
     }
-
+    // A reduction to tridiagonal form is backward stable in the norm of G only: it fixes a kept
+    // vector to an angle of a few eps |T| / gap, whatever the size of its eigenvalue.  Where a
+    // gap among the kept eigenvalues is too small for the angle the storage type needs (a
+    // strongly graded spectrum such as sigma_i = i^-1.5 over 128 directions), the Jacobi solve,
+    // which works to an accuracy relative to each eigenvalue, takes over at once.
+    __syncthreads();
+    {
+      int tight = 0;
+      if (wg == 0 && j < r - 1) tight = (lamv[j] - lamv[j + 1]) < tol.gap_min * lamv[0];
+      if (__syncthreads_or(tight)) {
+        ok = false;
+        if (tid == 0) s_why |= kWhyGap;
+      }
+    }
+    float* Vc = vs;        // current vectors
+    float* Vn = work;      // next (over the twisted-factorisation buffers once they are free)
+    if (ok || route == kRouteTridiag) {
     // ---- 4. twisted factorisation ---------------------------------------------------------------
     // The pivots of the two triangular factorisations of T - lambda I are ratios of consecutive
     // minors: q+_i = p_{i+1} / p_i with the leading minors p of the Sturm recurrence, and
@@ -661,11 +679,9 @@ __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const 
       reinterpret_cast<float4*>(Gsm)[e] = g;
     }
 
-    // ---- 6. V <- V (I - (V^T V - I) / 2) while V^T V - I is above the rounding level -----------
+    // ---- 6. orthogonalisation passes while V^T V - I is above the rounding level ---------------
     // Column-parallel: lane = column(s) c, c + 32; a warp takes RP / NW rows a of E.
     constexpr int AW = RP / NW;
-    float* Vc = vs;        // current vectors
-    float* Vn = work;      // next (the twisted-factorisation buffers are free now)
     for (;;) {
       float acc[NE][AW];
 #pragma unroll
@@ -715,14 +731,26 @@ __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const 
       __syncthreads();
       const float em = s_emax;
       if (em <= tol.ortho) break;                       // orthonormal to rounding
-      if (passes == 6 || !(em <= 0.5f)) { ok = false; if (tid == 0) s_why |= kWhyOrtho; break; }
+      if (passes == 6 || !(em <= 0.98f)) { ok = false; if (tid == 0) s_why |= kWhyOrtho; break; }
       ++passes;
-      // rows i of V' for this warp: D / NW of them; lane = column(s)
-      float ecol[NE][RP];
+      // One pass of Gram-Schmidt against the ORIGINAL earlier columns (larger eigenvalues, the
+      // better determined vectors): v_c <- (v_c - sum_{a<c} E_ac v_a) / |.|.  A later column never
+      // changes an earlier one, so a poorly separated pair cannot damage its neighbours; for
+      // two vectors the pass is exact, for more it converges quadratically like the symmetric
+      // form.  Rows i of V' for this warp: D / NW of them; lane = column(s).
+      float ecol[NE][RP], scol[NE];
 #pragma unroll
-      for (int h = 0; h < NE; ++h)
+      for (int h = 0; h < NE; ++h) {
+        const int c = 32 * h + lane;
+        float nn = 1.f;
 #pragma unroll
-        for (int a = 0; a < RP; ++a) ecol[h][a] = Em[a * RP + 32 * h + lane];
+        for (int a = 0; a < RP; ++a) {
+          const float e = Em[a * RP + c];
+          ecol[h][a] = a < c ? e : 0.f;
+          nn += a < c ? -e * e : (a == c ? e : 0.f);
+        }
+        scol[h] = rsqrtf(fmaxf(nn, 1e-6f));
+      }
       for (int i = warp; i < D; i += NW) {
         float o[NE];
 #pragma unroll
@@ -738,7 +766,7 @@ __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const 
         }
 #pragma unroll
         for (int h = 0; h < NE; ++h)
-          Vn[i * RP + 32 * h + lane] = fmaf(-0.5f, o[h], Vc[i * RP + 32 * h + lane]);
+          Vn[i * RP + 32 * h + lane] = (Vc[i * RP + 32 * h + lane] - o[h]) * scol[h];
       }
       __syncthreads();
       float* t = Vc; Vc = Vn; Vn = t;
@@ -824,6 +852,8 @@ __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const 
       }
       ok = __syncthreads_and(good) && ok;
     }
+
+    }   // the gaps allow the tridiagonal route
 
     if (ok || route == kRouteTridiag) {
       // singular values (non-increasing: a Rayleigh quotient may pass its neighbour by a rounding
@@ -1157,8 +1187,10 @@ cudaError_t launch_eig_tridiag(int B, int d, int r, solar_dtype_t dt, int route,
   TriTol tol;
   if (dt == SOLAR_BF16) {
     tol.eps_vec = 1e-3f; tol.floor_rel = 64.f * kUnit; tol.ortho = 4e-6f; tol.sweep_stop = 1e-3f;
+    tol.gap_min = 4.f * kUnit / 1e-2f;      // angle 1e-2: outputs are rounded to bf16 (2^-9)
   } else {
     tol.eps_vec = 1e-5f; tol.floor_rel = 32.f * kUnit; tol.ortho = 2e-6f; tol.sweep_stop = 1e-5f;
+    tol.gap_min = 4.f * kUnit / 1e-3f;
   }
   const bool wide = r > 32;
   switch (d) {
