@@ -152,8 +152,9 @@ cudaError_t launch_t(int B, int d, int r, const float* S, const float* V, const 
   const T* v = static_cast<const T*>(Wv);
 #define SOLAR_PREP(DD)                                                                          \
   {                                                                                             \
-    cudaError_t e = cudaFuncSetAttribute(attn_prepare_kernel<T, DD>,                            \
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+    static bool limits_set[kMaxDevicesCached] = {};                                             \
+    cudaError_t e = set_kernel_limits(reinterpret_cast<const void*>(&attn_prepare_kernel<T, DD>), \
+                                      (size_t)(2 * DD * DD + 2 * DD * 64) * sizeof(float), limits_set); \
     if (e != cudaSuccess) return e;                                                             \
     e = launch_pdl(attn_prepare_kernel<T, DD>, dim3(B, 2), dim3(kPrepThreads), smem, st, S, V, q, k, v, \
                    scale, r, ws, lay);                                                           \

@@ -278,8 +278,9 @@ cudaError_t launch_d(int B, int M, int r, const void* C, unsigned flags, void* O
   ok = ok && encode_tmap_bf16_3d(&tmV, ws + lay.vpk_off, kTokenSlots, 2 * D, (uint64_t)B, kTokenSlots * 2, pu,
                                  kTokenSlots, D);
   if (!ok) return cudaErrorInvalidValue;
-  cudaError_t e = cudaFuncSetAttribute(attn_umma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)Cfg::smem(kTokenSlots));
+  static bool limits_set[kMaxDevicesCached] = {};
+  const cudaError_t e = set_kernel_limits(reinterpret_cast<const void*>(&attn_umma_kernel<D>), Cfg::smem(kTokenSlots),
+                                          limits_set);
   if (e != cudaSuccess) return e;
   const dim3 grid((M + kRows - 1) / kRows, B), block(128);
   return launch_pdl(attn_umma_kernel<D>, grid, block, Cfg::smem(np), st, tmC, tmO, tmT, tmV, r, flags,

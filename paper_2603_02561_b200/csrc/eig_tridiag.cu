@@ -1157,16 +1157,10 @@ cudaError_t launch_tri(int B, int r, int route, int sweep_cap, TriTol tol, const
                        const int* gram_status, int splits, float* gsum, float* S, float* V, int* info,
                        int* route_taken, const FuseArgs& fa, cudaStream_t st) {
   using L = TriSmem<D, RP>;
-  static bool attr_set[64] = {};
-  int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
+  static bool limits_set[kMaxDevicesCached] = {};
+  const cudaError_t e = set_kernel_limits(reinterpret_cast<const void*>(&eig_tridiag_kernel<D, RP>), L::BYTES,
+                                          limits_set);
   if (e != cudaSuccess) return e;
-  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-    e = cudaFuncSetAttribute(eig_tridiag_kernel<D, RP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)L::BYTES);
-    if (e != cudaSuccess) return e;
-    if (dev >= 0 && dev < 64) attr_set[dev] = true;
-  }
   return launch_pdl(eig_tridiag_kernel<D, RP>, dim3(B), dim3(TriCfg<D>::NT), L::BYTES, st, gpart, gram_status,
                     splits, gsum, r, route, sweep_cap, tol, S, V, info, route_taken, fa);
 }

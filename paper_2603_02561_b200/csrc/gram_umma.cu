@@ -147,8 +147,8 @@ cudaError_t launch_d(int B, int N, const void* H, float* gpart, int* status, con
   if (!encode_tmap_bf16_3d(&tmap, H, D, (uint64_t)N, (uint64_t)B, (uint64_t)D * 2, (uint64_t)N * D * 2, 64,
                            kTileRows))
     return cudaErrorInvalidValue;
-  cudaError_t e = cudaFuncSetAttribute(gram_umma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)Cfg::SMEM);   // per device, cheap next to the launch
+  static bool limits_set[kMaxDevicesCached] = {};
+  const cudaError_t e = set_kernel_limits(reinterpret_cast<const void*>(&gram_umma_kernel<D>), Cfg::SMEM, limits_set);
   if (e != cudaSuccess) return e;
   const dim3 grid(plan.splits, B), block(128);
   return launch_pdl(gram_umma_kernel<D>, grid, block, Cfg::SMEM, st, tmap, gpart, status, N,

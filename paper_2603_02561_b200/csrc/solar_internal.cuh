@@ -190,6 +190,26 @@ bool attn_umma_supported(int d, solar_dtype_t dt);
 cudaError_t launch_attn_umma(int B, int M, int d, int r, const void* C, unsigned flags, void* O,
                              const char* ws, const AttnWs& lay, bool early_c, cudaStream_t st);
 
+// ---- per-kernel launch limits -----------------------------------------------------------------
+// Raises a kernel's dynamic shared-memory limit and asks for the largest shared-memory carve-out
+// (an SM keeps ONE carve-out at a time: kernels of several requests share an SM only if they
+// agree on it, and none of these kernels lives on L1), once per kernel and device: `done` is
+// the call site's own table.  A lost race between host threads only repeats the two calls.
+constexpr int kMaxDevicesCached = 64;
+inline cudaError_t set_kernel_limits(const void* func, size_t smem_bytes, bool (&done)[kMaxDevicesCached]) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const bool cached = dev >= 0 && dev < kMaxDevicesCached;
+  if (cached && done[dev]) return cudaSuccess;
+  e = cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(func, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared);
+  if (e != cudaSuccess) return e;
+  if (cached) done[dev] = true;
+  return cudaSuccess;
+}
+
 // ---- programmatic dependent launch ---------------------------------------------------
 // The four kernels of a forward pass run back to back on one stream.  Launched with this
 // attribute, a kernel may start while its predecessor is still draining; it does whatever
