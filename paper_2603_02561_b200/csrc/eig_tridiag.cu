@@ -123,13 +123,15 @@ __device__ __forceinline__ void tri_stage(float (&a)[TriCfg<D>::RPT][TriCfg<D>::
                                           float (&xc)[TriCfg<D>::CPT], float* __restrict__ hv,
                                           float* __restrict__ xpre, float* __restrict__ tpart,
                                           float* __restrict__ pvp, float* __restrict__ dg, float* __restrict__ eo,
-                                          float* __restrict__ betas, int tid) {
+                                          float* __restrict__ betas, int tid, float& tr_rest, float& tr_comp, float stop_tr,
+                                          float stop_x2, int r, int& k_stop) {
   using C = TriCfg<D>;
   constexpr int NW = C::NW, RPT = C::RPT, NG = C::NG, SS = C::SS;
   constexpr int G0 = S;                                               // first live column group
   constexpr int Q0 = (S * SS >= 31) ? (S * SS - 31) / 32 + 1 : 0;     // first live row slot
   constexpr int K1 = ((S + 1) * SS < D - 2) ? (S + 1) * SS : D - 2;
   const int lane = tid & 31, warp = tid >> 5;
+  if (k_stop >= 0) return;
 #pragma unroll 1
   for (int k = S * SS; k < K1; ++k) {
     const int k1 = k + 1, par = k & 1, q1 = k1 >> 5, l1 = k1 & 31;
@@ -156,6 +158,20 @@ __device__ __forceinline__ void tri_stage(float (&a)[TriCfg<D>::RPT][TriCfg<D>::
     // makes p, w and the update vanish, and the step still hands on column k+1.
     const bool reflect = tail2 > 1e-35f;
     const float s2 = fmaf(x1, x1, tail2);
+    // Rank-revealing stop: once the rows below k carry a negligible trace (G is positive
+    // semi-definite, so that bounds every entry of the block) and row k hardly couples to them,
+    // T ends at row k.  A history of low rank -- the premise of the method -- then costs its rank
+    // in Householder steps, and every later phase works on the shorter T.
+    {                                    // tr_rest -= dk, compensated (the trace is ~10^7 stop thresholds)
+      const float y = -dk - tr_comp, t = tr_rest + y;
+      tr_comp = (t - tr_rest) - y;
+      tr_rest = t;
+    }
+    if (k1 >= r && tr_rest <= stop_tr && s2 <= stop_x2) {
+      if (tid == 0) { dg[k] = dk; eo[k] = 0.f; betas[k] = 0.f; }
+      k_stop = k;
+      return;
+    }
     const float nrm = s2 * rsqrt_acc(fmaxf(s2, 1e-37f));
     const float alpha = reflect ? -copysignf(nrm, x1) : x1;
     const float vk1 = reflect ? x1 - alpha : 0.f;
@@ -242,13 +258,13 @@ __device__ __forceinline__ void tri_stage(float (&a)[TriCfg<D>::RPT][TriCfg<D>::
 // whichever sign the hardware gives it.
 template <int D, int CH>
 __device__ __forceinline__ void sturm(const float* __restrict__ dg, const float* __restrict__ e2s,
-                                      const float (&x)[CH], int (&cnt)[CH]) {
+                                      const float (&x)[CH], int (&cnt)[CH], int nb4) {
   float p[CH], q[CH];
   unsigned n[CH];
 #pragma unroll
   for (int h = 0; h < CH; ++h) { p[h] = 1.f; q[h] = 0.f; n[h] = 0; }
 #pragma unroll 4
-  for (int ib = 0; ib < D / 4; ++ib) {
+  for (int ib = 0; ib < nb4; ++ib) {
     const float4 d4 = *reinterpret_cast<const float4*>(dg + 4 * ib);
     const float4 e4 = *reinterpret_cast<const float4*>(e2s + 4 * ib);
     const float dd[4] = {d4.x, d4.y, d4.z, d4.w}, ee[4] = {e4.x, e4.y, e4.z, e4.w};
@@ -280,6 +296,8 @@ struct TriTol {
   float floor_rel;   // residuals below floor_rel * theta_1 are at the rounding level of fp32
   float ortho;       // largest |V^T V - I| entry that needs no further orthogonalisation
   float gap_min;     // smallest gap between kept eigenvalues, relative to the largest, the route is trusted with
+  float stop_trace;  // the reduction stops once the remaining rows' trace is below this fraction of trace(G) ...
+  float stop_couple; // ... and the current row couples to them by less than this fraction of it
   float sweep_stop;  // of the Jacobi fallback
 };
 
@@ -331,39 +349,35 @@ __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const 
     int lost = 0;
     for (int s = tid; s < splits; s += NT) lost |= (gram_status[b * splits + s] != kGramStatusOk);
     int bad = 0;
-    // fp32 sums in a fixed order (GW slices at a time, pairwise within the group); all loads of a
-    // group, for two elements, are issued before the first add: the loop is bound by their latency
-    static_assert((D * D / 4) % (2 * NT) == 0, "two elements per thread and trip");
-    for (int e = tid; e < D * D / 4; e += 2 * NT) {
-      constexpr int GW = 8;
-      float4 acc[2] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
-      for (int s = 0; s < splits; s += GW) {
-        float4 v[2][GW];
+    // fp32 sums in slice order.  A thread owns EPT 16-byte elements; the loads of SC slices for all
+    // of them are issued before the first add: the phase is bound by their latency.
+    constexpr int EPT = D * D / 4 / NT;
+    constexpr int SC = (EPT >= 16) ? 2 : (EPT >= 8) ? 3 : 8;
+    static_assert(EPT * NT * 4 == D * D, "whole elements");
+    float4 acc[EPT];
 #pragma unroll
-        for (int h = 0; h < 2; ++h)
+    for (int u = 0; u < EPT; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s0 = 0; s0 < splits; s0 += SC) {
+      float4 v[SC][EPT];
 #pragma unroll
-          for (int u = 0; u < GW; ++u)
-            v[h][u] = (s + u < splits) ? __ldg(gp + (size_t)(s + u) * (D * D / 4) + e + h * NT)
-                                       : make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int c = 0; c < SC; ++c)
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        for (int u = 0; u < EPT; ++u)
+          v[c][u] = (s0 + c < splits) ? __ldg(gp + (size_t)(s0 + c) * (D * D / 4) + tid + u * NT)
+                                      : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-          for (int w = GW / 2; w >= 1; w >>= 1)
+      for (int c = 0; c < SC; ++c)
 #pragma unroll
-            for (int u = 0; u < w; ++u) {
-              v[h][u].x += v[h][u + w].x; v[h][u].y += v[h][u + w].y;
-              v[h][u].z += v[h][u + w].z; v[h][u].w += v[h][u + w].w;
-            }
-          acc[h].x += v[h][0].x; acc[h].y += v[h][0].y; acc[h].z += v[h][0].z; acc[h].w += v[h][0].w;
+        for (int u = 0; u < EPT; ++u) {
+          acc[u].x += v[c][u].x; acc[u].y += v[c][u].y; acc[u].z += v[c][u].z; acc[u].w += v[c][u].w;
         }
-      }
+    }
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const int eh = e + h * NT;
-        bad |= !(isfinite(acc[h].x) && isfinite(acc[h].y) && isfinite(acc[h].z) && isfinite(acc[h].w));
-        *reinterpret_cast<float4*>(Gs + (eh / (D / 4)) * LD + (eh % (D / 4)) * 4) = acc[h];
-        reinterpret_cast<float4*>(gout)[eh] = acc[h];   // the residual check and the fallback read it back
-      }
+    for (int u = 0; u < EPT; ++u) {
+      const int eh = tid + u * NT;
+      bad |= !(isfinite(acc[u].x) && isfinite(acc[u].y) && isfinite(acc[u].z) && isfinite(acc[u].w));
+      *reinterpret_cast<float4*>(Gs + (eh / (D / 4)) * LD + (eh % (D / 4)) * 4) = acc[u];
+      reinterpret_cast<float4*>(gout)[eh] = acc[u];   // the residual check and the fallback read it back
     }
     if (tid < 4) s_flags[tid] = 0;
     if (tid == 0) s_why = 0;
@@ -401,6 +415,7 @@ __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const 
   int passes = 0;
   if (route != kRouteFull && gmax > 0.f) {
     // ---- 2. Householder tridiagonalisation, the matrix in registers ---------------------------
+    int k_stop = -1;                     // step at which the reduction stopped early (uniform), or -1
     {
       float a[RPT][CPT], xr[RPT], xc[CPT];
 #pragma unroll
@@ -420,37 +435,46 @@ __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const 
       for (int e = tid; e < D * D / 4; e += NT) reinterpret_cast<float4*>(hv)[e] = make_float4(0.f, 0.f, 0.f, 0.f);
       for (int e = tid; e < 2 * D; e += NT) xpre[e] = 0.f;
       __syncthreads();
-      tri_stage<D, 0>(a, xr, xc, hv, xpre, tpart, pvp, dg, eo, betas, tid);
-      tri_stage<D, 1>(a, xr, xc, hv, xpre, tpart, pvp, dg, eo, betas, tid);
+      const float trs = (float)((double)sc * s_trace);
+      float tr_rest = trs, tr_comp = 0.f;
+      const float stop_tr = trs * tol.stop_trace, stop_x2 = (trs * tol.stop_couple) * (trs * tol.stop_couple);
+      tri_stage<D, 0>(a, xr, xc, hv, xpre, tpart, pvp, dg, eo, betas, tid, tr_rest, tr_comp, stop_tr, stop_x2, r, k_stop);
+      tri_stage<D, 1>(a, xr, xc, hv, xpre, tpart, pvp, dg, eo, betas, tid, tr_rest, tr_comp, stop_tr, stop_x2, r, k_stop);
       if constexpr (NG > 2) {
-        tri_stage<D, 2>(a, xr, xc, hv, xpre, tpart, pvp, dg, eo, betas, tid);
-        tri_stage<D, 3>(a, xr, xc, hv, xpre, tpart, pvp, dg, eo, betas, tid);
+        tri_stage<D, 2>(a, xr, xc, hv, xpre, tpart, pvp, dg, eo, betas, tid, tr_rest, tr_comp, stop_tr, stop_x2, r, k_stop);
+        tri_stage<D, 3>(a, xr, xc, hv, xpre, tpart, pvp, dg, eo, betas, tid, tr_rest, tr_comp, stop_tr, stop_x2, r, k_stop);
       }
-      // the last 2 x 2 block: xr holds column D-2
-      if (warp == 0) {
+      if (k_stop < 0) {
+        // the last 2 x 2 block: xr holds column D-2
+        if (warp == 0) {
 #pragma unroll
-        for (int q = 0; q < RPT; ++q) {
-          if (lane + 32 * q == D - 2) dg[D - 2] = xr[q];
-          if (lane + 32 * q == D - 1) eo[D - 2] = xr[q];
+          for (int q = 0; q < RPT; ++q) {
+            if (lane + 32 * q == D - 2) dg[D - 2] = xr[q];
+            if (lane + 32 * q == D - 1) eo[D - 2] = xr[q];
+          }
+          if (lane == 0) { eo[D - 1] = 0.f; betas[D - 2] = 0.f; betas[D - 1] = 0.f; }
         }
-        if (lane == 0) { eo[D - 1] = 0.f; betas[D - 2] = 0.f; betas[D - 1] = 0.f; }
+        if (warp == NW - 1 && lane == 31) dg[D - 1] = a[RPT - 1][CPT - 1];
       }
-      if (warp == NW - 1 && lane == 31) dg[D - 1] = a[RPT - 1][CPT - 1];
     }
+    // T has `de` rows (all D unless the reduction stopped early), padded with zero rows to a multiple of 4
+    const int de = k_stop >= 0 ? k_stop + 1 : D, de4 = (de + 3) & ~3;
+    const int kb = k_stop >= 0 ? k_stop : D - 2;            // reflectors 0 .. kb-1 exist
+    if (tid < de4 - de) { dg[de + tid] = 0.f; eo[de + tid] = 0.f; }
     __syncthreads();
 
     // ---- 3. Gershgorin interval, floored squares, trace; multisection --------------------------
     if (warp == 0) {
       float lo = 3.0e38f, hi = -3.0e38f, tr = 0.f;
-      for (int i = lane; i < D; i += 32) {
-        const float rad = fabsf(eo[i]) + (i > 0 ? fabsf(eo[i - 1]) : 0.f);   // eo[D-1] = 0
+      for (int i = lane; i < de; i += 32) {
+        const float rad = fabsf(eo[i]) + (i > 0 ? fabsf(eo[i - 1]) : 0.f);   // eo[de-1] = 0
         lo = fminf(lo, dg[i] - rad); hi = fmaxf(hi, dg[i] + rad);
         tr += dg[i];
       }
       lo = -warp_max(-lo); hi = warp_max(hi); tr = warp_sum(tr);
       const float tn = fmaxf(fabsf(lo), fabsf(hi));
       const float fl = (tn * 1.4901161e-08f) * (tn * 1.4901161e-08f);         // (2^-26 |T|)^2
-      for (int i = lane; i < D; i += 32) e2s[i] = i > 0 ? fmaxf(eo[i - 1] * eo[i - 1], fl) : 0.f;
+      for (int i = lane; i < de4; i += 32) e2s[i] = i > 0 ? fmaxf(eo[i - 1] * eo[i - 1], fl) : 0.f;
       if (lane == 0) {
         const float span = hi - lo;
         s_lo = lo - 1e-6f * span - 1e-30f; s_hi = hi + 1e-6f * span + 1e-30f; s_trT = tr;
@@ -469,7 +493,7 @@ __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const 
       constexpr int STEPS = (P >= 8) ? 9 : 12;                   // (P + 1)^STEPS >= 2^27
       static_assert(2 * NE * P * 32 <= RP * RP, "flags fit in the E region");
       unsigned char* flag = reinterpret_cast<unsigned char*>(Em);   // [2][NE][P][32]: count(point) > target
-      const int target = D - 1 - jj;      // lambda_(jj-th largest) >= x  <=>  #(eigenvalues < x) <= target
+      const int target = de4 - 1 - jj;    // lambda_(jj-th largest) >= x  <=>  #(eigenvalues < x) <= target
       float lo = s_lo, hi = s_hi;
 #pragma unroll 1
       for (int step = 0; step < STEPS; ++step) {
@@ -478,7 +502,7 @@ __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const 
         int cnt[CH];
 #pragma unroll
         for (int h = 0; h < CH; ++h) x[h] = fmaf((float)(wg * CH + h + 1), w, lo);
-        sturm<D, CH>(dg, e2s, x, cnt);
+        sturm<D, CH>(dg, e2s, x, cnt, de4 >> 2);
         unsigned char* fl = flag + (((step & 1) * NE + gi) * P) * 32;
 #pragma unroll
         for (int h = 0; h < CH; ++h) fl[(wg * CH + h) * 32 + lane] = cnt[h] > target;
@@ -525,7 +549,7 @@ __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const 
       if (wg == 0) {
         float pf = 1.f, pfo = 0.f;                              // p_i, p_{i-1}
 #pragma unroll 8
-        for (int t = 0; t < D; ++t) {
+        for (int t = 0; t < de; ++t) {
           const float nf = fmaf(dg[t] - lam, pf, -(e2s[t] * pfo));
           float qf = __fdividef(nf, pf);
           qf = (fabsf(qf) >= pfl) ? qf : -pfl;                   // also catches NaN
@@ -541,8 +565,8 @@ __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const 
       if (wg == WB) {
         float pb = 1.f, pbo = 0.f;                              // t_{i+1}, t_{i+2}
 #pragma unroll 8
-        for (int t = 0; t < D; ++t) {
-          const int ib = D - 1 - t;
+        for (int t = 0; t < de; ++t) {
+          const int ib = de - 1 - t;
           const float nb = fmaf(dg[ib] - lam, pb, -((t > 0 ? e2s[ib + 1] : 0.f) * pbo));
           float qb = __fdividef(nb, pb);
           qb = (fabsf(qb) >= pfl) ? qb : -pfl;
@@ -560,19 +584,19 @@ __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const 
     {
       // gamma_i = q+_i + q-_i - (d_i - lambda) over my range of i; the multipliers
       // z_i = -(e_i / q+_i) z_{i+1} going up, z_i = -(e_{i-1} / q-_i) z_{i-1} going down
-      constexpr int IR = D / WG;
+      const int IR = (de + WG - 1) / WG, i1 = min((wg + 1) * IR, de);
       float best = 3.0e38f;
-      int kb = 0;
+      int kbest = 0;
 #pragma unroll 8
-      for (int i = wg * IR; i < (wg + 1) * IR; ++i) {
+      for (int i = wg * IR; i < i1; ++i) {
         const float qf = tf[i * RP + j], qb = tb[i * RP + j];
         const float gam = fabsf((qf + qb) - (dg[i] - lam));
-        if (gam < best) { best = gam; kb = i; }
+        if (gam < best) { best = gam; kbest = i; }
         tf[i * RP + j] = -__fdividef(eo[i], qf);
         tb[i * RP + j] = i > 0 ? -__fdividef(eo[i - 1], qb) : 0.f;
       }
       part[wg * RP + j] = best;
-      reinterpret_cast<int*>(part)[(NW + wg) * RP + j] = kb;
+      reinterpret_cast<int*>(part)[(NW + wg) * RP + j] = kbest;
     }
     __syncthreads();
     int kt = 0;
@@ -592,7 +616,7 @@ __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const 
       if (wg == 0) {
         float zu = 1.f, ss = 0.f;
 #pragma unroll 8
-        for (int iu = D - 2; iu >= 0; --iu) {
+        for (int iu = de - 2; iu >= 0; --iu) {
           const float mu = tf[iu * RP + j];
           zu = (iu < kt) ? zu * mu : 1.f;
           ss = fmaf(zu, (iu < kt) ? zu : 0.f, ss);
@@ -604,7 +628,7 @@ __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const 
       if (wg == WB) {
         float zd = 1.f, ss = 0.f;
 #pragma unroll 8
-        for (int t = 1; t < D; ++t) {
+        for (int t = 1; t < de; ++t) {
           const float md = tb[t * RP + j];
           zd = (t > kt) ? zd * md : 1.f;
           ss = fmaf(zd, (t > kt) ? zd : 0.f, ss);
@@ -638,10 +662,10 @@ __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const 
         for (int u = 0; u < RB; ++u) {
           const int i = qt * RB + u;
           const float upv = tf[i * RP + jc], dnv = tb[i * RP + jc];
-          z[u] = (i < ktj ? upv : i > ktj ? dnv : 1.f) * zn;
+          z[u] = i < de ? (i < ktj ? upv : i > ktj ? dnv : 1.f) * zn : 0.f;
         }
 #pragma unroll 2
-        for (int k = D - 3; k >= 0; --k) {
+        for (int k = kb - 1; k >= 0; --k) {
           const float beta = betas[k];
           const float4* h4 = reinterpret_cast<const float4*>(hv + k * D + qt * RB);
           float4 h[RB / 4];
@@ -1182,9 +1206,11 @@ cudaError_t launch_eig_tridiag(int B, int d, int r, solar_dtype_t dt, int route,
   if (dt == SOLAR_BF16) {
     tol.eps_vec = 1e-3f; tol.floor_rel = 64.f * kUnit; tol.ortho = 4e-6f; tol.sweep_stop = 1e-3f;
     tol.gap_min = 4.f * kUnit / 1e-2f;      // angle 1e-2: outputs are rounded to bf16 (2^-9)
+    tol.stop_trace = 1.9073486e-06f; tol.stop_couple = 2.3841858e-07f;     // 2^-19, 2^-22
   } else {
     tol.eps_vec = 1e-5f; tol.floor_rel = 32.f * kUnit; tol.ortho = 2e-6f; tol.sweep_stop = 1e-5f;
     tol.gap_min = 4.f * kUnit / 1e-3f;
+    tol.stop_trace = 1.1920929e-07f; tol.stop_couple = 2.9802322e-08f;     // 2^-23, 2^-25
   }
   const bool wide = r > 32;
   switch (d) {
