@@ -166,21 +166,27 @@ solar_status_t solar_svd_attention_fused(int B, int M, int N, int d, int r, sola
  * checked on its own; argument meaning and rules are those given above.
  * ------------------------------------------------------------------------- */
 
-/* Number of row-slices each H_b is cut into by solar_gram_partials (>= 1). */
+/* Number of partial Gram matrices solar_gram_partials leaves per user (>= 1; usually 1), and
+ * the number of row slices (CTAs, status words) per user behind them (a multiple of it). */
 int solar_gram_splits(int B, int N, int d, solar_dtype_t dt);
+int solar_gram_slices(int B, int N, int d, solar_dtype_t dt);
 
-/* Streaming pass over H: slice s of user b contributes the d x d partial Gram
- *   P[b,s] = sum over the rows n of slice s of h_n h_n^T        (fp32)
- * stored at ((float*)workspace)[(b*splits + s)*d*d ...], row-major; the kernel's
- * per-slice status words follow the partials (read by solar_eig_from_partials).
- * H_b^T H_b (the matrix whose eigenvectors are V of Eq. 9) is the sum over s.
- * bf16 storage with d = 64 or 128 and N >= 128 runs on the tensor cores (TMA tiles,
- * tcgen05.mma, fp32 accumulation in tensor memory); other shapes use FFMA. */
+/* Streaming pass over H.  Every H_b is cut into row slices (one CTA each); partial p of
+ * user b is the sum of h_n h_n^T over the rows n of its group of slices (fp32), stored at
+ *   ((float*)workspace)[(b*P + p)*d*d ...],  P = solar_gram_splits(),  row-major;
+ * the kernel's per-slice status words follow the partials (read by
+ * solar_eig_from_partials).  H_b^T H_b (the matrix whose eigenvectors are V of Eq. 9) is
+ * the sum over p.  bf16 storage with d = 64 or 128 and N >= 128 runs on the tensor cores
+ * (TMA tiles, tcgen05.mma, fp32 accumulation in tensor memory; the CTAs of up to eight
+ * slices form a thread-block cluster and add up their results through distributed shared
+ * memory, so P is 1 unless more than eight slices are the better cut); other shapes use
+ * FFMA with one partial per slice. */
 solar_status_t solar_gram_partials(int B, int N, int d, solar_dtype_t dt, const void* H,
                                    void* workspace, size_t workspace_bytes, void* stream);
 
 /* Sums the partial Grams in slice order and diagonalises; writes S, V, info.  The summed
- * matrices [B,d,d] fp32 are left in the workspace behind the status words. */
+ * matrices [B,d,d] fp32 are left in the workspace (behind the status words, or in place of
+ * the partials where a user has only one). */
 solar_status_t solar_eig_from_partials(int B, int N, int d, int r, solar_dtype_t dt,
                                        float* S, float* V, int* info,
                                        void* workspace, size_t workspace_bytes, void* stream);
@@ -304,7 +310,7 @@ solar_status_t solar_factored_softmax_attention_fwd(int B, int M, int N, int d, 
  *   - Same arguments, outputs, info bits and rules as solar_lowrank_factor,
  *     minus US and the workspace.  Calls no cudaMalloc / cudaFree and no
  *     allocating library routine.
- *   - Sizes whose scratch need, B * solar_gram_splits(B,N,d,dt) * d*d*4 bytes,
+ *   - Sizes whose scratch need, solar_workspace_bytes(B, 0, N, d, r, dt) bytes,
  *     exceeds the array return SOLAR_ERR_WORKSPACE before anything is launched
  *     (the headline shape B=16, N=10240, d=64 needs 2.25 MiB).
  *   - The first call on each device looks up the array's device address (with

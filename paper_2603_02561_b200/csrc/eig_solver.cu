@@ -333,7 +333,7 @@ __device__ __forceinline__ int ritz_jacobi(float* Tb, float* Wb, int p, float th
 
 template <int D>
 __global__ void __launch_bounds__(EigCfg<D>::THREADS, 1)
-eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status, int splits, int r,
+eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status, int parts, int splits, int r,
            int p, int route, int sweep_cap, int force_iters, EigTol tol, float* __restrict__ S,
            float* __restrict__ V, int* __restrict__ info, int* __restrict__ route_taken) {
   using Cfg = EigCfg<D>;
@@ -351,7 +351,7 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
   pdl_wait();          // everything below reads what the Gram kernel wrote
 
   // ---- G = sum of the slices' partial Grams, in slice order -----------------
-  const float4* gp = reinterpret_cast<const float4*>(gpart + (size_t)b * splits * D * D);
+  const float4* gp = reinterpret_cast<const float4*>(gpart + (size_t)b * parts * D * D);
   // a Gram CTA whose bounded wait ran out leaves a code other than kGramStatusOk
   int lost = 0;
   for (int s = tid; s < splits; s += NT) lost |= (gram_status[b * splits + s] != kGramStatusOk);
@@ -362,11 +362,11 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
     // All loads of a group are issued before the first add: the loop is bound by their latency.
     constexpr int GW = (D == 128) ? 8 : 16;      // 1024 threads leave 64 registers each at d = 128
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s = 0; s < splits; s += GW) {
+    for (int s = 0; s < parts; s += GW) {
       float4 v[GW];
 #pragma unroll
       for (int u = 0; u < GW; ++u)
-        v[u] = (s + u < splits) ? __ldg(gp + (size_t)(s + u) * (D * D / 4) + e)
+        v[u] = (s + u < parts) ? __ldg(gp + (size_t)(s + u) * (D * D / 4) + e)
                                 : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
       for (int h = GW / 2; h >= 1; h >>= 1)
@@ -619,14 +619,14 @@ eig_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status,
 
 template <int D>
 cudaError_t launch_d(int B, int r, int p, int route, int sweep_cap, int force_iters, EigTol tol, const float* gpart,
-                     const int* gram_status, int splits, float* S, float* V, int* info,
+                     const int* gram_status, int parts, int splits, float* S, float* V, int* info,
                      int* route_taken, cudaStream_t st) {
   using Cfg = EigCfg<D>;
   if (p > Cfg::PMAX) p = 0;
   cudaError_t e = cudaFuncSetAttribute(eig_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)Cfg::SMEM);
   if (e != cudaSuccess) return e;
-  return launch_pdl(eig_kernel<D>, dim3(B), dim3(Cfg::THREADS), Cfg::SMEM, st, gpart, gram_status, splits,
+  return launch_pdl(eig_kernel<D>, dim3(B), dim3(Cfg::THREADS), Cfg::SMEM, st, gpart, gram_status, parts, splits,
                     r, p, route, sweep_cap, force_iters, tol, S, V, info, route_taken);
 }
 
@@ -641,12 +641,12 @@ int eig_subspace_dim(int d, int r) {
 }
 
 cudaError_t launch_eig(int B, int d, int r, solar_dtype_t dt, int route, int sweep_cap, int force_iters,
-                       const float* gpart, const int* gram_status, int splits, float* gsum, float* S,
+                       const float* gpart, const int* gram_status, int parts, int splits, float* gsum, float* S,
                        float* V, int* info, int* route_taken, cudaStream_t st) {
   if (sweep_cap <= 0 || sweep_cap > kMaxSweeps) sweep_cap = kMaxSweeps;
   // AUTO and TRIDIAG: the tridiagonal route (with the Jacobi solve behind it in AUTO)
   if (route == SOLAR_ROUTE_AUTO || route == SOLAR_ROUTE_TRIDIAG)
-    return launch_eig_tridiag(B, d, r, dt, route, sweep_cap, gpart, gram_status, splits, gsum, S, V, info,
+    return launch_eig_tridiag(B, d, r, dt, route, sweep_cap, gpart, gram_status, parts, splits, gsum, S, V, info,
                               route_taken, nullptr, st);
   EigTol tol;
   if (dt == SOLAR_BF16) {
@@ -656,9 +656,9 @@ cudaError_t launch_eig(int B, int d, int r, solar_dtype_t dt, int route, int swe
   }
   const int p = eig_subspace_dim(d, r);
   switch (d) {
-    case 32: return launch_d<32>(B, r, p, route, sweep_cap, force_iters, tol, gpart, gram_status, splits, S, V, info, route_taken, st);
-    case 64: return launch_d<64>(B, r, p, route, sweep_cap, force_iters, tol, gpart, gram_status, splits, S, V, info, route_taken, st);
-    case 128: return launch_d<128>(B, r, p, route, sweep_cap, force_iters, tol, gpart, gram_status, splits, S, V, info, route_taken, st);
+    case 32: return launch_d<32>(B, r, p, route, sweep_cap, force_iters, tol, gpart, gram_status, parts, splits, S, V, info, route_taken, st);
+    case 64: return launch_d<64>(B, r, p, route, sweep_cap, force_iters, tol, gpart, gram_status, parts, splits, S, V, info, route_taken, st);
+    case 128: return launch_d<128>(B, r, p, route, sweep_cap, force_iters, tol, gpart, gram_status, parts, splits, S, V, info, route_taken, st);
     default: return cudaErrorInvalidValue;
   }
 }

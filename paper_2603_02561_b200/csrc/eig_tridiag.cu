@@ -306,7 +306,7 @@ struct TriTol {
 // shared memory ([D][rp], rp = r rounded up to 4, zero in the padding) and true is returned.
 template <int D, int RP>
 __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const int* __restrict__ gram_status,
-                                         int splits, float* __restrict__ gsum, int r, int route, int sweep_cap,
+                                         int parts, int splits, float* __restrict__ gsum, int r, int route, int sweep_cap,
                                          const TriTol& tol, bool want_vs, float* __restrict__ S,
                                          float* __restrict__ V, int* __restrict__ info,
                                          int* __restrict__ route_taken) {
@@ -343,9 +343,10 @@ __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const 
 
   // ---- 1. G = sum of the slices' partial Grams, in a fixed order -----------------------------
   float* Gs = work;    // [D][LD] staging copy
-  float* gout = gsum + (size_t)b * D * D;
+  // the summed matrix in global memory: a user's only partial as it is, else written below
+  const float* gout = parts == 1 ? gpart + (size_t)b * D * D : gsum + (size_t)b * D * D;
   {
-    const float4* gp = reinterpret_cast<const float4*>(gpart + (size_t)b * splits * D * D);
+    const float4* gp = reinterpret_cast<const float4*>(gpart + (size_t)b * parts * D * D);
     int lost = 0;
     for (int s = tid; s < splits; s += NT) lost |= (gram_status[b * splits + s] != kGramStatusOk);
     int bad = 0;
@@ -357,13 +358,13 @@ __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const 
     float4 acc[EPT];
 #pragma unroll
     for (int u = 0; u < EPT; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s0 = 0; s0 < splits; s0 += SC) {
+    for (int s0 = 0; s0 < parts; s0 += SC) {
       float4 v[SC][EPT];
 #pragma unroll
       for (int c = 0; c < SC; ++c)
 #pragma unroll
         for (int u = 0; u < EPT; ++u)
-          v[c][u] = (s0 + c < splits) ? __ldg(gp + (size_t)(s0 + c) * (D * D / 4) + tid + u * NT)
+          v[c][u] = (s0 + c < parts) ? __ldg(gp + (size_t)(s0 + c) * (D * D / 4) + tid + u * NT)
                                       : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
       for (int c = 0; c < SC; ++c)
@@ -377,7 +378,7 @@ __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const 
       const int eh = tid + u * NT;
       bad |= !(isfinite(acc[u].x) && isfinite(acc[u].y) && isfinite(acc[u].z) && isfinite(acc[u].w));
       *reinterpret_cast<float4*>(Gs + (eh / (D / 4)) * LD + (eh % (D / 4)) * 4) = acc[u];
-      reinterpret_cast<float4*>(gout)[eh] = acc[u];   // the residual check and the fallback read it back
+      if (parts > 1) reinterpret_cast<float4*>(gsum + (size_t)b * D * D)[eh] = acc[u];   // the residual check and the fallback read it back
     }
     if (tid < 4) s_flags[tid] = 0;
     if (tid == 0) s_why = 0;
@@ -1163,11 +1164,11 @@ __device__ __forceinline__ void prepare_epilogue(float* __restrict__ sm, int b, 
 
 template <int D, int RP>
 __global__ void __launch_bounds__(TriCfg<D>::NT, 1)
-eig_tridiag_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status, int splits,
+eig_tridiag_kernel(const float* __restrict__ gpart, const int* __restrict__ gram_status, int parts, int splits,
                    float* __restrict__ gsum, int r, int route, int sweep_cap, TriTol tol,
                    float* __restrict__ S, float* __restrict__ V, int* __restrict__ info,
                    int* __restrict__ route_taken, FuseArgs fa) {
-  const bool vs_ready = eig_user<D, RP>(gpart, gram_status, splits, gsum, r, route, sweep_cap, tol, fa.mode != 0, S, V,
+  const bool vs_ready = eig_user<D, RP>(gpart, gram_status, parts, splits, gsum, r, route, sweep_cap, tol, fa.mode != 0, S, V,
                                         info, route_taken);
   if (fa.mode != 0) {
     extern __shared__ __align__(16) float smem[];
@@ -1178,7 +1179,7 @@ eig_tridiag_kernel(const float* __restrict__ gpart, const int* __restrict__ gram
 
 template <int D, int RP>
 cudaError_t launch_tri(int B, int r, int route, int sweep_cap, TriTol tol, const float* gpart,
-                       const int* gram_status, int splits, float* gsum, float* S, float* V, int* info,
+                       const int* gram_status, int parts, int splits, float* gsum, float* S, float* V, int* info,
                        int* route_taken, const FuseArgs& fa, cudaStream_t st) {
   using L = TriSmem<D, RP>;
   static bool limits_set[kMaxDevicesCached] = {};
@@ -1186,13 +1187,13 @@ cudaError_t launch_tri(int B, int r, int route, int sweep_cap, TriTol tol, const
                                           limits_set);
   if (e != cudaSuccess) return e;
   return launch_pdl(eig_tridiag_kernel<D, RP>, dim3(B), dim3(TriCfg<D>::NT), L::BYTES, st, gpart, gram_status,
-                    splits, gsum, r, route, sweep_cap, tol, S, V, info, route_taken, fa);
+                    parts, splits, gsum, r, route, sweep_cap, tol, S, V, info, route_taken, fa);
 }
 
 }  // namespace
 
 cudaError_t launch_eig_tridiag(int B, int d, int r, solar_dtype_t dt, int route, int sweep_cap,
-                               const float* gpart, const int* gram_status, int splits, float* gsum,
+                               const float* gpart, const int* gram_status, int parts, int splits, float* gsum,
                                float* S, float* V, int* info, int* route_taken, const EigFuse* fuse,
                                cudaStream_t st) {
   FuseArgs fa = {};
@@ -1215,13 +1216,13 @@ cudaError_t launch_eig_tridiag(int B, int d, int r, solar_dtype_t dt, int route,
   const bool wide = r > 32;
   switch (d) {
     case 32:
-      return launch_tri<32, 32>(B, r, route, sweep_cap, tol, gpart, gram_status, splits, gsum, S, V, info, route_taken, fa, st);
+      return launch_tri<32, 32>(B, r, route, sweep_cap, tol, gpart, gram_status, parts, splits, gsum, S, V, info, route_taken, fa, st);
     case 64:
-      return wide ? launch_tri<64, 64>(B, r, route, sweep_cap, tol, gpart, gram_status, splits, gsum, S, V, info, route_taken, fa, st)
-                  : launch_tri<64, 32>(B, r, route, sweep_cap, tol, gpart, gram_status, splits, gsum, S, V, info, route_taken, fa, st);
+      return wide ? launch_tri<64, 64>(B, r, route, sweep_cap, tol, gpart, gram_status, parts, splits, gsum, S, V, info, route_taken, fa, st)
+                  : launch_tri<64, 32>(B, r, route, sweep_cap, tol, gpart, gram_status, parts, splits, gsum, S, V, info, route_taken, fa, st);
     case 128:
-      return wide ? launch_tri<128, 64>(B, r, route, sweep_cap, tol, gpart, gram_status, splits, gsum, S, V, info, route_taken, fa, st)
-                  : launch_tri<128, 32>(B, r, route, sweep_cap, tol, gpart, gram_status, splits, gsum, S, V, info, route_taken, fa, st);
+      return wide ? launch_tri<128, 64>(B, r, route, sweep_cap, tol, gpart, gram_status, parts, splits, gsum, S, V, info, route_taken, fa, st)
+                  : launch_tri<128, 32>(B, r, route, sweep_cap, tol, gpart, gram_status, parts, splits, gsum, S, V, info, route_taken, fa, st);
     default: return cudaErrorInvalidValue;
   }
 }

@@ -55,7 +55,7 @@ solar_status_t solar_lowrank_factor_static(int B, int M, int N, int d, int r, so
     return solar_lowrank_factor(B, 0, N, d, r, dt, H, S, V, nullptr, info, nullptr, 0, stream);
   }
   if (B == 0) return SOLAR_OK;
-  if (solar::factor_ws_bytes(B, N, d) > kStaticScratchBytes) return SOLAR_ERR_WORKSPACE;
+  if (solar::factor_ws_bytes(B, N, d, dt) > kStaticScratchBytes) return SOLAR_ERR_WORKSPACE;
   void* scratch = nullptr;
   const solar_status_t st = scratch_for_current_device(&scratch);
   if (st != SOLAR_OK) return st;

@@ -6,8 +6,14 @@
 // through a ring of shared-memory stages with TMA (128-byte swizzle, zero fill past row
 // N, so ragged tails add nothing); a single thread issues tcgen05.mma with the SAME tile
 // as both operands -- H^T as an MN-major A and H as an MN-major B, K = the 128 rows --
-// accumulating the d x d result in tensor memory; all four warps then move it to global
-// memory.  H is read from HBM exactly once and never passes through registers.
+// accumulating the d x d result in tensor memory.  H is read from HBM exactly once and never
+// passes through registers.
+//
+// The CTAs of up to eight slices of a user form a thread-block cluster: each lays its
+// accumulator down in its own shared memory, and after a cluster barrier every CTA adds up
+// one share of the matrix over all of them through distributed shared memory (plain loads, in
+// rank order: the sum is reproducible) and stores it.  A user so leaves splits / cluster
+// partial matrices in global memory -- one in the usual case -- instead of one per slice.
 #include "sm100_ptx.cuh"
 #include "solar_internal.cuh"
 
@@ -32,7 +38,7 @@ template <int D> struct GramCfg {
 template <int D>
 __global__ void __launch_bounds__(128, 1)
 gram_umma_kernel(const __grid_constant__ CUtensorMap tmap, float* __restrict__ gpart,
-                 int* __restrict__ status, int N, int chunk_rows, int splits) {
+                 int* __restrict__ status, int N, int chunk_rows, int splits, int cluster) {
   using Cfg = GramCfg<D>;
   constexpr int STAGES = Cfg::STAGES;
   extern __shared__ uint8_t smem_raw[];
@@ -105,15 +111,16 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tmap, float* __restrict__ g
   }
   __syncwarp();
 
-  // ---- epilogue: tensor memory -> P[b,s] (row-major fp32) ------------------------------
+  // ---- epilogue: tensor memory -> shared memory -> sum over the cluster -> global ----------
   const bool done = ptx::mbar_wait(&accum_bar, 0, err, kErrEpilogue);
   pdl_trigger();       // only the epilogue is left: the next kernel may start launching
   __syncwarp();
   ptx::tc_fence_after_sync();
-  float* out = gpart + ((size_t)b * splits + s) * D * D;
-  // nothing is written before the previous kernel on the stream (it may still be reading this
-  // workspace) has completed
-  pdl_wait();
+  // the accumulator as a row-major fp32 matrix over the ring (every tile has been consumed);
+  // the row pitch D + 4 keeps the 16-byte stores of a warp's 32 rows off each other's banks
+  constexpr int LDR = D + 4;
+  float* red = reinterpret_cast<float*>(tiles);
+  static_assert((size_t)D * LDR * sizeof(float) <= (size_t)STAGES * Cfg::TILE_BYTES, "the matrix fits over the ring");
   if (done && *err == 0) {
     // M = 128: accumulator row i sits in lane i.  M = 64: rows 16q .. 16q+15 sit in lanes
     // 32q .. 32q+15 (each warp reaches only its own 32-lane quarter).
@@ -125,7 +132,7 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tmap, float* __restrict__ g
       ptx::tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + c0, v);
       ptx::tmem_ld_wait();
       if (has_row) {
-        float4* dst = reinterpret_cast<float4*>(out + (size_t)row * D + c0);
+        float4* dst = reinterpret_cast<float4*>(red + (size_t)row * LDR + c0);
 #pragma unroll
         for (int q = 0; q < 8; ++q)
           dst[q] = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
@@ -137,6 +144,32 @@ gram_umma_kernel(const __grid_constant__ CUtensorMap tmap, float* __restrict__ g
   __syncthreads();
   if (warp == 1) ptx::tmem_dealloc(tmem, D);
   if (tid == 0) status[b * splits + s] = (s_err == 0) ? kGramStatusOk : s_err;
+  // Every CTA of the cluster reaches the two cluster barriers, whatever happened above (a lost
+  // wait is reported through the status word; the sum of that user is then not used).
+  if (cluster > 1) ptx::cluster_sync();
+  // nothing is written before the previous kernel on the stream (it may still be reading this
+  // workspace) has completed
+  pdl_wait();
+  {
+    const int rank = s % cluster;
+    float* out = gpart + ((size_t)b * (splits / cluster) + s / cluster) * D * D;
+    // this CTA's share of the matrix: 16-byte elements rank, rank + cluster, ...
+    for (int e = rank * 128 + tid; e < D * D / 4; e += cluster * 128) {
+      const int row = e / (D / 4), c4 = e % (D / 4);
+      const float* src = red + (size_t)row * LDR + 4 * c4;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (cluster > 1) {
+        for (int q = 0; q < cluster; ++q) {
+          const float4 t = ptx::ld_cluster_f4(src, q);
+          acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+        }
+      } else {
+        acc = *reinterpret_cast<const float4*>(src);
+      }
+      reinterpret_cast<float4*>(out)[e] = acc;
+    }
+  }
+  if (cluster > 1) ptx::cluster_sync();      // nobody leaves while its matrix is still being read
 }
 
 template <int D>
@@ -151,8 +184,16 @@ cudaError_t launch_d(int B, int N, const void* H, float* gpart, int* status, con
   const cudaError_t e = set_kernel_limits(reinterpret_cast<const void*>(&gram_umma_kernel<D>), Cfg::SMEM, limits_set);
   if (e != cudaSuccess) return e;
   const dim3 grid(plan.splits, B), block(128);
-  return launch_pdl(gram_umma_kernel<D>, grid, block, Cfg::SMEM, st, tmap, gpart, status, N,
-                    plan.chunk_tiles * kTileRows, plan.splits);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = Cfg::SMEM; cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = (unsigned)plan.cluster; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = plan.cluster > 1 ? 2 : 1;
+  return cudaLaunchKernelEx(&cfg, gram_umma_kernel<D>, tmap, gpart, status, N, plan.chunk_tiles * kTileRows,
+                            plan.splits, plan.cluster);
 }
 
 }  // namespace

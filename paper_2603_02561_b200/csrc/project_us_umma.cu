@@ -201,7 +201,7 @@ project_us_umma_kernel(const __grid_constant__ CUtensorMap tmap, const float* __
 template <int D>
 cudaError_t launch_d(int B, int N, int r, const void* H, const float* V, void* US, cudaStream_t st) {
   using Cfg = UsCfg<D>;
-  const GramPlan plan = gram_plan(B, N);
+  const GramPlan plan = slice_plan(B, N);
   CUtensorMap tmap;
   if (!encode_tmap_bf16_3d(&tmap, H, D, (uint64_t)N, (uint64_t)B, (uint64_t)D * 2, (uint64_t)N * D * 2, 64,
                            kTileRows))

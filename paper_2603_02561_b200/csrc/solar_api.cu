@@ -45,7 +45,7 @@ solar_status_t attn_apply_impl(int B, int M, int d, int r, solar_dtype_t dt, con
 }
 
 // Workspace of the fused forward call: the factorization's, then the attention's.
-size_t fused_attn_offset(int B, int N, int d) { return align_up(factor_ws_bytes(B, N, d), 256); }
+size_t fused_attn_offset(int B, int N, int d, solar_dtype_t dt) { return align_up(factor_ws_bytes(B, N, d, dt), 256); }
 
 }  // namespace
 
@@ -64,14 +64,19 @@ const char* solar_status_string(solar_status_t st) {
 
 size_t solar_workspace_bytes(int B, int M, int N, int d, int r, solar_dtype_t dt) {
   if (check_dims(B, M, N, d, r, dt) != SOLAR_OK) return 0;
-  const size_t f = factor_ws_bytes(B, N, d), a = attn_ws_bytes(B, d, r);
+  const size_t f = factor_ws_bytes(B, N, d, dt), a = attn_ws_bytes(B, d, r);
   const size_t need = f > a ? f : a;
   return need ? need : 256;
 }
 
 int solar_gram_splits(int B, int N, int d, solar_dtype_t dt) {
   if (check_dims(B, 0, N, d, 1, dt) != SOLAR_OK) return 0;
-  return gram_plan(B, N).splits;
+  return gram_plan(B, N, gram_is_clustered(N, d, dt)).parts;
+}
+
+int solar_gram_slices(int B, int N, int d, solar_dtype_t dt) {
+  if (check_dims(B, 0, N, d, 1, dt) != SOLAR_OK) return 0;
+  return gram_plan(B, N, gram_is_clustered(N, d, dt)).splits;
 }
 
 solar_status_t solar_gram_partials(int B, int N, int d, solar_dtype_t dt, const void* H,
@@ -79,10 +84,10 @@ solar_status_t solar_gram_partials(int B, int N, int d, solar_dtype_t dt, const 
   SOLAR_TRY(check_dims(B, 0, N, d, 1, dt));
   if (B == 0) return SOLAR_OK;
   SOLAR_TRY(check_ptr(H));
-  SOLAR_TRY(check_ws(workspace, workspace_bytes, factor_ws_bytes(B, N, d)));
-  const GramPlan plan = gram_plan(B, N);
+  SOLAR_TRY(check_ws(workspace, workspace_bytes, factor_ws_bytes(B, N, d, dt)));
+  const GramPlan plan = gram_plan(B, N, gram_is_clustered(N, d, dt));
   float* gpart = static_cast<float*>(workspace);
-  int* status = reinterpret_cast<int*>(static_cast<char*>(workspace) + gram_status_offset(B, N, d));
+  int* status = reinterpret_cast<int*>(static_cast<char*>(workspace) + gram_status_offset(B, N, d, dt));
   const cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (gram_umma_supported(N, d, dt)) return from_cuda(launch_gram_umma(B, N, d, H, gpart, status, plan, st));
   return from_cuda(launch_gram_simt(B, N, d, dt, H, gpart, status, plan, st));
@@ -100,13 +105,13 @@ solar_status_t solar_eig_from_partials_ex(int B, int N, int d, int r, solar_dtyp
   if (info != nullptr && (reinterpret_cast<uintptr_t>(info) & 3u)) return SOLAR_ERR_INVALID_ARG;
   if (route_taken != nullptr && (reinterpret_cast<uintptr_t>(route_taken) & 3u))
     return SOLAR_ERR_INVALID_ARG;
-  SOLAR_TRY(check_ws(workspace, workspace_bytes, factor_ws_bytes(B, N, d)));
-  const GramPlan plan = gram_plan(B, N);
+  SOLAR_TRY(check_ws(workspace, workspace_bytes, factor_ws_bytes(B, N, d, dt)));
+  const GramPlan plan = gram_plan(B, N, gram_is_clustered(N, d, dt));
   const int* status =
-      reinterpret_cast<const int*>(static_cast<const char*>(workspace) + gram_status_offset(B, N, d));
-  float* gsum = reinterpret_cast<float*>(static_cast<char*>(workspace) + gram_sum_offset(B, N, d));
+      reinterpret_cast<const int*>(static_cast<const char*>(workspace) + gram_status_offset(B, N, d, dt));
+  float* gsum = reinterpret_cast<float*>(static_cast<char*>(workspace) + gram_sum_offset(B, N, d, dt));
   return from_cuda(launch_eig(B, d, r, dt, base_route, sweep_cap, force_iters, static_cast<const float*>(workspace),
-                              status, plan.splits, gsum, S, V, info, route_taken,
+                              status, plan.parts, plan.splits, gsum, S, V, info, route_taken,
                               static_cast<cudaStream_t>(stream)));
 }
 
@@ -138,7 +143,7 @@ solar_status_t solar_lowrank_factor(int B, int M, int N, int d, int r, solar_dty
   SOLAR_TRY(check_ptr(V));
   if (US != nullptr) SOLAR_TRY(check_ptr(US));
   if (info != nullptr && (reinterpret_cast<uintptr_t>(info) & 3u)) return SOLAR_ERR_INVALID_ARG;
-  SOLAR_TRY(check_ws(workspace, workspace_bytes, factor_ws_bytes(B, N, d)));
+  SOLAR_TRY(check_ws(workspace, workspace_bytes, factor_ws_bytes(B, N, d, dt)));
   SOLAR_TRY(solar_gram_partials(B, N, d, dt, H, workspace, workspace_bytes, stream));
   SOLAR_TRY(solar_eig_from_partials(B, N, d, r, dt, S, V, info, workspace, workspace_bytes, stream));
   if (US != nullptr) SOLAR_TRY(solar_project_us(B, N, d, r, dt, H, V, US, stream));
@@ -200,7 +205,7 @@ solar_status_t solar_svd_attention_fwd(int B, int M, int N, int d, int r, solar_
 
 size_t solar_fused_workspace_bytes(int B, int M, int N, int d, int r, solar_dtype_t dt) {
   if (check_dims(B, M, N, d, r, dt) != SOLAR_OK) return 0;
-  return fused_attn_offset(B, N, d) + align_up(attn_ws_bytes(B, d, r), 256);
+  return fused_attn_offset(B, N, d, dt) + align_up(attn_ws_bytes(B, d, r), 256);
 }
 
 solar_status_t solar_svd_attention_fused(int B, int M, int N, int d, int r, solar_dtype_t dt,
@@ -222,16 +227,16 @@ solar_status_t solar_svd_attention_fused(int B, int M, int N, int d, int r, sola
   SOLAR_TRY(check_ws(workspace, workspace_bytes, solar_fused_workspace_bytes(B, M, N, d, r, dt)));
   const cudaStream_t st = static_cast<cudaStream_t>(stream);
   char* ws = static_cast<char*>(workspace);
-  char* attn_ws = ws + fused_attn_offset(B, N, d);
+  char* attn_ws = ws + fused_attn_offset(B, N, d, dt);
   // streaming pass over H (the first kernel of the call: it waits for what ran before)
-  SOLAR_TRY(solar_gram_partials(B, N, d, dt, H, workspace, factor_ws_bytes(B, N, d), stream));
+  SOLAR_TRY(solar_gram_partials(B, N, d, dt, H, workspace, factor_ws_bytes(B, N, d, dt), stream));
   // eigensolve; every user's CTA ends with that user's factor-token projections
-  const GramPlan plan = gram_plan(B, N);
-  const int* status = reinterpret_cast<const int*>(ws + gram_status_offset(B, N, d));
-  float* gsum = reinterpret_cast<float*>(ws + gram_sum_offset(B, N, d));
+  const GramPlan plan = gram_plan(B, N, gram_is_clustered(N, d, dt));
+  const int* status = reinterpret_cast<const int*>(ws + gram_status_offset(B, N, d, dt));
+  float* gsum = reinterpret_cast<float*>(ws + gram_sum_offset(B, N, d, dt));
   const EigFuse fuse = {Wq, Wk, Wv, scale, attn_ws};
   SOLAR_TRY(from_cuda(launch_eig_tridiag(B, d, r, dt, SOLAR_ROUTE_AUTO, kMaxSweeps, reinterpret_cast<const float*>(ws),
-                                         status, plan.splits, gsum, S, V, info, nullptr, &fuse, st)));
+                                         status, plan.parts, plan.splits, gsum, S, V, info, nullptr, &fuse, st)));
   if (M == 0) return SOLAR_OK;
   return attn_apply_impl(B, M, d, r, dt, C, flags, O, attn_ws, true, st);
 }

@@ -19,49 +19,83 @@ constexpr int kMaxSweeps = 16;      // Jacobi sweep cap
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline size_t elem_size(solar_dtype_t dt) { return dt == SOLAR_BF16 ? 2 : 4; }
 
-// How each H_b is cut into row slices for the streaming Gram pass.  The cost
-// model is waves(B*S CTAs over the SMs) x (tiles per slice + fixed per-CTA cost).
+// How each H_b is cut into row slices for a streaming pass (one CTA per user and slice).  The
+// cost model is waves(B*S CTAs over the SMs) x (tiles per slice + fixed per-CTA cost).
 struct GramPlan {
   int tiles;        // ceil(N / kGramTileRows)
   int chunk_tiles;  // tiles per slice
   int splits;       // slices per user (all non-empty)
+  int cluster;      // slices whose CTAs form one thread-block cluster and add up their results on chip
+  int parts;        // partial Gram matrices per user that reach global memory: splits / cluster
 };
 
-inline GramPlan gram_plan(int B, int N) {
+inline long slice_cost(int B, int tiles, int s, int* s_eff_out, int* chunk_out) {
+  const int chunk = (tiles + s - 1) / s;
+  const int s_eff = (tiles + chunk - 1) / chunk;
+  const long waves = ((long)B * s_eff + kNumSMs - 1) / kNumSMs;
+  *s_eff_out = s_eff; *chunk_out = chunk;
+  return waves * (chunk + 2);
+}
+
+inline GramPlan slice_plan(int B, int N) {
   GramPlan p;
   p.tiles = (N + kGramTileRows - 1) / kGramTileRows;
-  int best_s = 1;
   long best_cost = -1;
   const int smax = p.tiles < kMaxSplits ? p.tiles : kMaxSplits;
+  p.splits = 1; p.chunk_tiles = p.tiles;
   for (int s = 1; s <= smax; ++s) {
-    const int chunk = (p.tiles + s - 1) / s;
-    const int s_eff = (p.tiles + chunk - 1) / chunk;
-    const long waves = ((long)B * s_eff + kNumSMs - 1) / kNumSMs;
-    const long cost = waves * (chunk + 2);
-    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_s = s_eff; }
+    int s_eff, chunk;
+    const long cost = slice_cost(B, p.tiles, s, &s_eff, &chunk);
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; p.splits = s_eff; p.chunk_tiles = chunk; }
   }
-  p.splits = best_s;
-  p.chunk_tiles = (p.tiles + best_s - 1) / best_s;
-  p.splits = (p.tiles + p.chunk_tiles - 1) / p.chunk_tiles;
+  p.cluster = 1;
+  p.parts = p.splits;
   return p;
 }
 
-// Workspace of the factorization: partial Grams [B][splits][d][d] fp32, then one status
-// word per (user, slice), written by every Gram CTA: kGramStatusOk, or the code of the
-// bounded device-side wait that ran out.
+// The plan of the tensor-core Gram kernel: the CTAs of up to eight slices of a user form a
+// cluster and reduce their accumulators through distributed shared memory, so a user leaves
+// splits / cluster partial matrices (one, whenever eight slices or fewer are the best cut).
+// Candidates are the slice counts a cluster can cover: 1 .. 8, then multiples of 8.
+constexpr int kMaxCluster = 8;
+inline GramPlan gram_plan(int B, int N, bool clustered) {
+  if (!clustered) return slice_plan(B, N);
+  GramPlan p;
+  p.tiles = (N + kGramTileRows - 1) / kGramTileRows;
+  long best_cost = -1;
+  const int smax = p.tiles < kMaxSplits ? p.tiles : kMaxSplits;
+  p.splits = 1; p.chunk_tiles = p.tiles;
+  for (int s = 1; s <= smax; ++s) {
+    int s_eff, chunk;
+    const long cost = slice_cost(B, p.tiles, s, &s_eff, &chunk);
+    if (s_eff > kMaxCluster && s_eff % kMaxCluster != 0) continue;
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; p.splits = s_eff; p.chunk_tiles = chunk; }
+  }
+  p.cluster = p.splits <= kMaxCluster ? p.splits : kMaxCluster;
+  p.parts = p.splits / p.cluster;
+  return p;
+}
+inline bool gram_is_clustered(int N, int d, solar_dtype_t dt) {
+  return dt == SOLAR_BF16 && (d == 64 || d == 128) && N >= kGramTileRows;   // the tensor-core kernel's shapes
+}
+
+// Workspace of the factorization: partial Grams [B][parts][d][d] fp32, then one status word per
+// (user, slice), written by every Gram CTA: kGramStatusOk, or the code of the bounded
+// device-side wait that ran out.
 constexpr int kGramStatusOk = 0x600D;
-inline size_t gram_status_offset(int B, int N, int d) {
-  const GramPlan p = gram_plan(B, N);
-  return align_up((size_t)B * p.splits * d * d * sizeof(float), 256);
+inline size_t gram_status_offset(int B, int N, int d, solar_dtype_t dt) {
+  const GramPlan p = gram_plan(B, N, gram_is_clustered(N, d, dt));
+  return align_up((size_t)B * p.parts * d * d * sizeof(float), 256);
 }
 // Behind the status words: the summed Gram matrices [B][d][d] fp32, written by the eigensolver
-// (its residual check and its Jacobi fallback read them back).
-inline size_t gram_sum_offset(int B, int N, int d) {
-  const GramPlan p = gram_plan(B, N);
-  return gram_status_offset(B, N, d) + align_up((size_t)B * p.splits * sizeof(int), 256);
+// when a user has more than one partial (its residual check and its Jacobi fallback read the
+// sum back; a single partial is the sum).
+inline size_t gram_sum_offset(int B, int N, int d, solar_dtype_t dt) {
+  const GramPlan p = gram_plan(B, N, gram_is_clustered(N, d, dt));
+  return gram_status_offset(B, N, d, dt) + align_up((size_t)B * p.splits * sizeof(int), 256);
 }
-inline size_t factor_ws_bytes(int B, int N, int d) {
-  return gram_sum_offset(B, N, d) + align_up((size_t)B * d * d * sizeof(float), 256);
+inline size_t factor_ws_bytes(int B, int N, int d, solar_dtype_t dt) {
+  return gram_sum_offset(B, N, d, dt) + align_up((size_t)B * d * d * sizeof(float), 256);
 }
 
 // Workspace of the attention call, per user (all segments 256-byte aligned):
@@ -146,8 +180,9 @@ cudaError_t launch_gram_simt(int B, int N, int d, solar_dtype_t dt, const void* 
 bool gram_umma_supported(int N, int d, solar_dtype_t dt);
 cudaError_t launch_gram_umma(int B, int N, int d, const void* H, float* gpart, int* status,
                              const GramPlan& plan, cudaStream_t st);
+// parts: partial Gram matrices per user; splits: status words per user
 cudaError_t launch_eig(int B, int d, int r, solar_dtype_t dt, int route, int sweep_cap, int force_iters,
-                       const float* gpart, const int* gram_status, int splits, float* gsum, float* S,
+                       const float* gpart, const int* gram_status, int parts, int splits, float* gsum, float* S,
                        float* V, int* info, int* route_taken, cudaStream_t st);
 // The eigensolver CTA of a user may end with that user's factor-token projections (Eq. 11):
 // weights in the storage type, the attention workspace of all users.
@@ -157,7 +192,7 @@ struct EigFuse {
   char* attn_ws;
 };
 cudaError_t launch_eig_tridiag(int B, int d, int r, solar_dtype_t dt, int route, int sweep_cap,
-                               const float* gpart, const int* gram_status, int splits, float* gsum,
+                               const float* gpart, const int* gram_status, int parts, int splits, float* gsum,
                                float* S, float* V, int* info, int* route_taken, const EigFuse* fuse,
                                cudaStream_t st);
 int eig_subspace_dim(int d, int r);

@@ -39,6 +39,7 @@ SIGNATURES = {
     "solar_svd_attention_fused": (_c_int, [_c_int] * 5 + [_c_int] + [_c_vp] * 5 + [_c_float, _c_uint] +
                                   [_c_vp] * 4 + [_c_vp, _c_size, _c_vp]),
     "solar_gram_splits": (_c_int, [_c_int] * 3 + [_c_int]),
+    "solar_gram_slices": (_c_int, [_c_int] * 3 + [_c_int]),
     "solar_gram_partials": (_c_int, [_c_int] * 3 + [_c_int, _c_vp, _c_vp, _c_size, _c_vp]),
     "solar_eig_from_partials": (_c_int, [_c_int] * 4 + [_c_int] + [_c_vp] * 3 + [_c_vp, _c_size, _c_vp]),
     "solar_eig_from_partials_ex": (_c_int, [_c_int] * 4 + [_c_int, _c_int] + [_c_vp] * 4 +
@@ -111,6 +112,10 @@ def workspace_bytes(B, M, N, d, r, dtype) -> int:
 
 def gram_splits(B, N, d, dtype) -> int:
     return int(lib().solar_gram_splits(B, N, d, dtype_code(dtype)))
+
+
+def gram_slices(B, N, d, dtype) -> int:
+    return int(lib().solar_gram_slices(B, N, d, dtype_code(dtype)))
 
 
 def alloc_workspace(B, M, N, d, r, dtype, device="cuda") -> torch.Tensor:

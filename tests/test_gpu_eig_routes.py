@@ -184,10 +184,11 @@ def test_lost_gram_slice_reaches_the_caller():
     tdt = torch.bfloat16
     H = ph.to_device(inp["H"], w.dtype)
     ws = solar.alloc_workspace(w.B, w.M, w.N, w.d, w.r, tdt)
-    splits = solar.gram_splits(w.B, w.N, w.d, tdt)
+    parts = solar.gram_splits(w.B, w.N, w.d, tdt)          # partial matrices per user
+    splits = solar.gram_slices(w.B, w.N, w.d, tdt)         # slices (CTAs, status words) per user
     solar.gram_partials(H, ws)
     torch.cuda.synchronize()
-    off = (w.B * splits * w.d * w.d * 4 + 255) // 256 * 256
+    off = (w.B * parts * w.d * w.d * 4 + 255) // 256 * 256
     status = ws[off: off + 4 * w.B * splits].view(torch.int32)
     assert torch.all(status == 0x600D)
     ref = {}
