@@ -187,6 +187,35 @@ def test_invariances():
     assert np.abs(s2 - math.sqrt(2) * s1).max() < 1e-11 and np.abs(V1 - V2).max() < 1e-10
 
 
+# ---- P8b: the power iteration of Algorithm 1 on a full-rank history -----------------------
+def test_randomized_svd_power_steps_contract_the_subspace_error():
+    """On a full-rank H with singular values sigma_i = 4 * 2^-i the range of H^T(H Omega) loses
+    the discarded directions by (sigma_{r+1} / sigma_r)^2 = 1/4 per power step (subspace
+    iteration with H^T H): the tangent of the largest principal angle between R and the true
+    top-r right subspace (LAPACK) must fall by that factor from n_iter to n_iter + 1.  A power
+    loop that does not run, or that applies anything but H^T H, leaves the band."""
+    rng = np.random.default_rng(21)
+    N, d, r = 80, 12, 4
+    U0, _ = np.linalg.qr(rng.standard_normal((N, d)))
+    V0, _ = np.linalg.qr(rng.standard_normal((d, d)))
+    sig = 4.0 * 0.5 ** np.arange(d)
+    H = (U0 * sig) @ V0.T
+    Vt = np.linalg.svd(H, full_matrices=False)[2]
+    Vtop, Vrest = Vt[:r].T, Vt[r:].T
+    Omega = rng.standard_normal((d, r))
+    tans = []
+    for n_iter in (0, 1, 2, 3):
+        _, R = o.randomized_svd(H, r, n_iter, Omega)
+        Qr, _ = np.linalg.qr(R)                          # R is orthonormal already; this only guards the test
+        # tan of the largest principal angle: largest singular value of (Vrest^T Q)(Vtop^T Q)^-1
+        tans.append(np.linalg.svd((Vrest.T @ Qr) @ np.linalg.inv(Vtop.T @ Qr), compute_uv=False)[0])
+    q2 = (sig[r] / sig[r - 1]) ** 2
+    assert tans[0] > 1e-3                                # no power step: a visibly wrong subspace
+    for a, b in zip(tans[:-1], tans[1:]):
+        assert q2 / 2 <= b / a <= q2 * 2, (tans, q2)
+    assert tans[1] < 0.6 * tans[0]                       # one step differs measurably from none
+
+
 # ---- P8: Algorithm 1 reaches the same factors on rank-r input ----------------------
 @pytest.mark.parametrize("n_iter", [0, 2])
 def test_randomized_svd_matches_on_low_rank(n_iter):
