@@ -228,7 +228,11 @@ solar_status_t solar_attn_apply(int B, int M, int d, int r, solar_dtype_t dt, co
  * dV^T V, the index order for which the formula is the derivative of the forward pass
  * (the appendix's expansion of the trace has the indices transposed, which flips the sign
  * of that term).  Evaluated as one more streaming pass over H:  dH_b = H_b K_b with
- * K_b = V Sigma^-1 [.] V^T, so U is never materialised.
+ * K_b = V Sigma^-1 [.] V^T, so U is never materialised.  For r < d this is the part of
+ * the gradient that acts within the kept subspace: the component of dV orthogonal to span(V)
+ * and the coupling to the discarded singular pairs are left out (the bias the paper bounds
+ * by |dV_orth|_F / sigma_r).  It is the exact gradient for r = d and for perturbations of
+ * the form U X V^T.
  *
  *   H   [B,N,d] dt  (in)   the histories given to solar_lowrank_factor
  *   S   [B,r]  f32  (in)   singular values,  V [B,d,r] f32 (in) right singular vectors
@@ -315,7 +319,8 @@ solar_status_t solar_factored_softmax_attention_fwd(int B, int M, int N, int d, 
  *     (the headline shape B=16, N=10240, d=64 needs 2.25 MiB).
  *   - The first call on each device looks up the array's device address (with
  *     that device current) and caches it; make that first call outside any
- *     stream capture.
+ *     stream capture.  The array is chosen by the CURRENT device: the device
+ *     that `stream` belongs to must be current when the call is made.
  *   - All calls on a device share the one array: it keeps whatever the last call
  *     left (every slice is fully overwritten before it is read, nothing needs
  *     zeroing), and two calls that overlap on the GPU -- different streams,

@@ -72,6 +72,15 @@ CONFIGS = {
     # online-serving shape of Table 3 (12,000 behaviours x 3000 candidates), rank ~ Figure 1
     "serve": Workload("serve", "bf16", 8, 12000, 64, 32, 3000, "spectrum", rank=32,
                       decay=1.0, seed_index=6),
+    # the same shape at the rank Figure 1 reads off a user sequence (27: not a multiple of 8 or 16)
+    "serve27": Workload("serve27", "bf16", 8, 12000, 64, 27, 3000, "spectrum", rank=27,
+                        decay=1.0, seed_index=7),
+    # offline evaluation shape of Table 3 (history 50, 120 candidates per request; many requests per
+    # batch): N < d, so the history has at most 50 directions, kept at rank 16 and 27
+    "offline16": Workload("offline16", "bf16", 128, 50, 64, 16, 120, "product_noise", rank=16,
+                          noise_var=1e-3, seed_index=8),
+    "offline27": Workload("offline27", "bf16", 128, 50, 64, 27, 120, "product_noise", rank=27,
+                          noise_var=1e-3, seed_index=9),
 }
 
 

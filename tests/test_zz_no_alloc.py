@@ -51,3 +51,25 @@ def test_static_scratch_variant_matches_workspace_variant_twice():
             tol = 1e-5 if w.dtype == "f32" else 1e-4      # the singular-value tolerance of the parity tests
             assert np.abs(s1 - s0).max() <= tol * s0.max(), (rep, w.name)
             assert np.abs(v1 - v0).max() <= tol, (rep, w.name)
+            # the same kernels in the same order on the same numbers: the bits agree as well
+            assert torch.equal(S0, S1) and torch.equal(V0, V1), (rep, w.name)
+
+
+@pytest.mark.gpu
+def test_static_scratch_variant_allocates_nothing():
+    """After the first call on the device (which looks up the array's address), a call leaves
+    both the caching allocator's books and the driver's free-memory figure where they were."""
+    w = wl.CONFIGS["c2"].with_(B=4, N=700, M=4)
+    inp = wl.generate(w)
+    H = ph.to_device(inp["H"], w.dtype)
+    S = torch.empty(w.B, w.r, device="cuda"); V = torch.empty(w.B, w.d, w.r, device="cuda")
+    info = torch.empty(w.B, dtype=torch.int32, device="cuda")
+    solar.lowrank_factor_static(H, w.r, S=S, V=V, info=info)          # first call: set-up
+    torch.cuda.synchronize()
+    before = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), torch.cuda.mem_get_info()[0])
+    for _ in range(3):
+        solar.lowrank_factor_static(H, w.r, S=S, V=V, info=info)
+    torch.cuda.synchronize()
+    after = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), torch.cuda.mem_get_info()[0])
+    assert before == after, (before, after)
+    assert (info == 0).all()
