@@ -45,14 +45,22 @@ L2_BYTES = 126 * 2 ** 20
 KERNELS_PER_STEP = {"fused": 3, "two_call": 4}   # gram, eigensolve (+ projections), [projections,] attention
 FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # 148 SMs x 128 FMA lanes x 2 flop at 1965 MHz
 SFU_TEXPS = 148 * 16 * 1.965e9 / 1e12              # 148 SMs x 16 special-function lanes at 1965 MHz
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
-# profiles/ (null once the kernel has changed since the capture)
-TRAFFIC = {
-    ("c3", "gram"): 20987904,        # profiles/gram_umma_c3.md
-    ("c3", "attn_apply"): 4628224,   # profiles/attn_umma_c3.md (O still in L2 when the kernel ends)
-    ("c3", "eig"): 2432000,          # profiles/eig_kernel_c3.md
-    ("c3", "attn_prepare"): 187136,  # profiles/attn_prepare_c3.md
-}
+def measured_traffic(workload: str, kernel: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture recorded in
+    the traffic file -- or None when there is no capture for this workload and kernel, or the
+    kernel's source has changed since the counters were taken."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        rec = json.load(open(path)).get(f"{workload}/{kernel}")
+        if rec is None:
+            return None
+        src = os.path.join(ROOT, rec["source"])
+        if hashlib.sha1(open(src, "rb").read()).hexdigest()[:16] != rec["source_sha1"]:
+            return None
+        return rec["dram_bytes_per_launch"]
+    except Exception:
+        return None
 
 
 def peaks():
@@ -143,12 +151,25 @@ def oracle_step(w: wl.Workload, users):
 
 
 def cpu_threads() -> int:
+    """Threads of the BLAS pool numpy's matrix products run on (the oracle's Jacobi loop itself
+    is Python-level and serial)."""
     try:
         from threadpoolctl import threadpool_info
         n = [p.get("num_threads", 1) for p in threadpool_info()]
         return max(n) if n else 1
     except Exception:
         return 1
+
+
+def oracle_step_single_thread(w: wl.Workload, users):
+    """The same with every BLAS pool limited to one thread: the condition of the paper's own
+    latency experiment (Section 5.2: CPU, a single thread)."""
+    try:
+        from threadpoolctl import threadpool_limits
+    except Exception:
+        return None
+    with threadpool_limits(limits=1):
+        return oracle_step(w, users)
 
 
 def run_reference(args, w: wl.Workload):
@@ -226,6 +247,9 @@ def main():
     ap.add_argument("--cpu-users", type=int, default=8, help="users in the cpu_baseline sample")
     ap.add_argument("--ref-users", type=int, default=2, help="users per step of --impl reference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--light", action="store_true",
+                    help="the forward path only (no backward / factored-exact sections, short timed region): "
+                         "what the profiler captures are taken on")
     ap.add_argument("--sweep", action="store_true",
                     help="the c5 sweep: one JSON line per (N, r) point, with a brute-force softmax "
                          "attention time on the host beside it")
@@ -268,7 +292,7 @@ def main():
                 print(json.dumps(line), flush=True)
             torch.cuda.empty_cache()
     else:
-        line = measure(args, w, torch, dist, solar, world, rank, local)
+        line = measure(args, w, torch, dist, solar, world, rank, local, light=args.light)
         if rank == 0:
             print(json.dumps(line), flush=True)
     if world > 1:
@@ -581,9 +605,10 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
         "attn_prepare": {"bound": "alu", "achieved": 6.0 * w.B * w.r * w.d * w.d / (stage_ms["attn_prepare"] * 1e-3) / 1e12,
                          "peak": FP32_ALU_TFLOPS, "unit": "TFLOP/s"},
     }
-    for v in per_kernel.values():
+    for k, v in per_kernel.items():
         v["frac"] = v["achieved"] / v["peak"]
-    traffic = TRAFFIC.get((w.name, dominant))
+        v["traffic"] = measured_traffic(w.name, k)
+    traffic = measured_traffic(w.name, dominant)
     roof = dict(per_kernel[dominant], kernel=dominant, traffic=traffic, peak_source=pk["source"])
     line = {
         "metric": "svd_attention_fwd_candidates_x_positions_per_sec",
@@ -631,9 +656,16 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
     if not args.no_cpu_baseline and world >= 1:
         users = list(range(min(w.B, args.cpu_users)))
         t = oracle_step(w, users)
+        one = users[:max(1, len(users) // 4)]
+        t1 = oracle_step_single_thread(w, one)
         line["cpu_baseline"] = {"value": len(users) * w.M * w.N / t, "unit": "pairs/s",
-                                "cores": cpu_threads(), "kind": "oracle", "seconds": t,
-                                "sample": f"{len(users)} of {w.B} users, all {w.M} candidates"}
+                                "cores": cpu_threads(), "host_cpus": os.cpu_count(), "kind": "oracle", "seconds": t,
+                                "sample": f"{len(users)} of {w.B} users, all {w.M} candidates",
+                                "note": "numpy fp64; the Jacobi sweeps are a Python loop, only its matrix "
+                                        "products use the BLAS pool of `cores` threads",
+                                "single_thread": None if t1 is None else {
+                                    "value": len(one) * w.M * w.N / t1, "unit": "pairs/s", "cores": 1, "seconds": t1,
+                                    "sample": f"{len(one)} of {w.B} users, all {w.M} candidates, BLAS pools limited to 1 thread"}}
     return line
 
 

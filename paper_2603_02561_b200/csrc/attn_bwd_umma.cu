@@ -38,18 +38,6 @@ template <int D> struct BwdCfg {
   }
 };
 
-__device__ __forceinline__ uint32_t swz(int row, int c) {
-  return (uint32_t)row * 128u + (uint32_t)((c ^ (row & 7)) << 4);
-}
-__device__ __forceinline__ float fast_exp2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<const uint32_t*>(&v);
-}
 // eight values as a bf16 high half and the bf16 of what the high half misses
 __device__ __forceinline__ void split8(const float* x, uint4& hi, uint4& lo) {
   uint32_t h[4], l[4];
@@ -58,8 +46,8 @@ __device__ __forceinline__ void split8(const float* x, uint4& hi, uint4& lo) {
     const float x0 = x[2 * q], x1 = x[2 * q + 1];
     const float h0 = __bfloat162float(__float2bfloat16_rn(x0));
     const float h1 = __bfloat162float(__float2bfloat16_rn(x1));
-    h[q] = pack_bf16(h0, h1);
-    l[q] = pack_bf16(x0 - h0, x1 - h1);
+    h[q] = ptx::pack_bf16(h0, h1);
+    l[q] = ptx::pack_bf16(x0 - h0, x1 - h1);
   }
   hi = make_uint4(h[0], h[1], h[2], h[3]);
   lo = make_uint4(l[0], l[1], l[2], l[3]);
@@ -195,7 +183,7 @@ attn_bwd_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_const
       float sum = 0.f;
 #pragma unroll
       for (int i = 0; i < kTokenSlots; ++i) {
-        p[i] = (i < r) ? fast_exp2((p[i] - mx) * 1.4426950408889634f) : 0.f;
+        p[i] = (i < r) ? ptx::fast_exp2((p[i] - mx) * 1.4426950408889634f) : 0.f;
         sum += p[i];
       }
       const float inv = 1.f / sum;
@@ -233,11 +221,11 @@ attn_bwd_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_const
         for (int c = 0; c < 4; ++c) {
           uint4 hi, lo;
           split8(&p[c0 + 8 * c], hi, lo);
-          *reinterpret_cast<uint4*>(sP + swz(tid, c0 / 8 + c)) = hi;
-          *reinterpret_cast<uint4*>(sP + kBoxBytes + swz(tid, c0 / 8 + c)) = lo;
+          *reinterpret_cast<uint4*>(sP + ptx::swz128(tid, c0 / 8 + c)) = hi;
+          *reinterpret_cast<uint4*>(sP + kBoxBytes + ptx::swz128(tid, c0 / 8 + c)) = lo;
           split8(&dsv[8 * c], hi, lo);
-          *reinterpret_cast<uint4*>(sD + swz(tid, c0 / 8 + c)) = hi;
-          *reinterpret_cast<uint4*>(sD + kBoxBytes + swz(tid, c0 / 8 + c)) = lo;
+          *reinterpret_cast<uint4*>(sD + ptx::swz128(tid, c0 / 8 + c)) = hi;
+          *reinterpret_cast<uint4*>(sD + kBoxBytes + ptx::swz128(tid, c0 / 8 + c)) = lo;
         }
       }
     }
@@ -299,11 +287,11 @@ attn_bwd_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_const
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         const uint4 w = make_uint4(
-            pack_bf16(__uint_as_float(v[8 * c + 0]), __uint_as_float(v[8 * c + 1])),
-            pack_bf16(__uint_as_float(v[8 * c + 2]), __uint_as_float(v[8 * c + 3])),
-            pack_bf16(__uint_as_float(v[8 * c + 4]), __uint_as_float(v[8 * c + 5])),
-            pack_bf16(__uint_as_float(v[8 * c + 6]), __uint_as_float(v[8 * c + 7])));
-        *reinterpret_cast<uint4*>(box + swz(tid, (c0 % 64) / 8 + c)) = w;
+            ptx::pack_bf16(__uint_as_float(v[8 * c + 0]), __uint_as_float(v[8 * c + 1])),
+            ptx::pack_bf16(__uint_as_float(v[8 * c + 2]), __uint_as_float(v[8 * c + 3])),
+            ptx::pack_bf16(__uint_as_float(v[8 * c + 4]), __uint_as_float(v[8 * c + 5])),
+            ptx::pack_bf16(__uint_as_float(v[8 * c + 6]), __uint_as_float(v[8 * c + 7])));
+        *reinterpret_cast<uint4*>(box + ptx::swz128(tid, (c0 % 64) / 8 + c)) = w;
       }
     }
     ptx::fence_proxy_async_smem();

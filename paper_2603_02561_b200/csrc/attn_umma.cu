@@ -40,28 +40,6 @@ template <int D> struct AttnCfg {
   static constexpr int TMEM_COLS = D;                             // scores (<= 64 columns), then the output (D)
 };
 
-// Byte offset of 16-byte chunk c of row `row` in a 128-byte-swizzled tile of 128-byte rows.
-__device__ __forceinline__ uint32_t swz(int row, int c) {
-  return (uint32_t)row * 128u + (uint32_t)((c ^ (row & 7)) << 4);
-}
-// The same for a 64-byte-swizzled tile of 64-byte rows (4 chunks per row; address bits 4-5 are
-// XORed with bits 7-8, i.e. with row / 2).
-__device__ __forceinline__ uint32_t swz64(int row, int c) {
-  return (uint32_t)row * 64u + (uint32_t)((c ^ ((row >> 1) & 3)) << 4);
-}
-
-// 2^x by the special-function unit (2 ulp; the probabilities are rounded to bf16 pairs anyway).
-__device__ __forceinline__ float fast_exp2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<const uint32_t*>(&v);
-}
-
 template <int D>
 __global__ void __launch_bounds__(128)
 attn_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmO,
@@ -170,7 +148,7 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
     float sum = 0.f;
 #pragma unroll
     for (int i = 0; i < kTokenSlots; ++i) {
-      p[i] = (i < r) ? fast_exp2((p[i] - mx) * 1.4426950408889634f) : 0.f;
+      p[i] = (i < r) ? ptx::fast_exp2((p[i] - mx) * 1.4426950408889634f) : 0.f;
       sum += p[i];
     }
     const float inv = 1.f / sum;
@@ -190,10 +168,10 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
         const float x0 = p[8 * c + 2 * q], x1 = p[8 * c + 2 * q + 1];
         const float h0 = __bfloat162float(__float2bfloat16_rn(x0));
         const float h1 = __bfloat162float(__float2bfloat16_rn(x1));
-        hi[q] = pack_bf16(h0, h1);
-        lo[q] = pack_bf16(x0 - h0, x1 - h1);
+        hi[q] = ptx::pack_bf16(h0, h1);
+        lo[q] = ptx::pack_bf16(x0 - h0, x1 - h1);
       }
-      const uint32_t off = p64 ? swz64(tid, c) : swz(tid, c);
+      const uint32_t off = p64 ? ptx::swz64(tid, c) : ptx::swz128(tid, c);
       *reinterpret_cast<uint4*>(sP + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
       *reinterpret_cast<uint4*>(sP + p_half + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
     }
@@ -237,11 +215,11 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_constant_
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
       const uint4 w = make_uint4(
-          pack_bf16(__uint_as_float(v[8 * c + 0]), __uint_as_float(v[8 * c + 1])),
-          pack_bf16(__uint_as_float(v[8 * c + 2]), __uint_as_float(v[8 * c + 3])),
-          pack_bf16(__uint_as_float(v[8 * c + 4]), __uint_as_float(v[8 * c + 5])),
-          pack_bf16(__uint_as_float(v[8 * c + 6]), __uint_as_float(v[8 * c + 7])));
-      *reinterpret_cast<uint4*>(box + swz(tid, (c0 % 64) / 8 + c)) = w;
+          ptx::pack_bf16(__uint_as_float(v[8 * c + 0]), __uint_as_float(v[8 * c + 1])),
+          ptx::pack_bf16(__uint_as_float(v[8 * c + 2]), __uint_as_float(v[8 * c + 3])),
+          ptx::pack_bf16(__uint_as_float(v[8 * c + 4]), __uint_as_float(v[8 * c + 5])),
+          ptx::pack_bf16(__uint_as_float(v[8 * c + 6]), __uint_as_float(v[8 * c + 7])));
+      *reinterpret_cast<uint4*>(box + ptx::swz128(tid, (c0 % 64) / 8 + c)) = w;
     }
   }
   ptx::fence_proxy_async_smem();

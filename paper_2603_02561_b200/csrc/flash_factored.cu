@@ -46,18 +46,6 @@ template <int D, int R> struct FlashCfg {
   static constexpr int TMEM_COLS = (D == 64) ? 256 : 512;
 };
 
-__device__ __forceinline__ uint32_t swz128(int row, int c) {   // 16-byte chunk c of a 128-byte swizzled row
-  return (uint32_t)row * 128u + (uint32_t)((c ^ (row & 7)) << 4);
-}
-__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
-  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<const uint32_t*>(&v);
-}
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
 // Writes R fp32 values of this thread's row as bf16 high and low halves into two swizzled
 // K-major tiles (hi at `dst`, lo one box further).
 template <int R>
@@ -69,11 +57,11 @@ __device__ __forceinline__ void store_hi_lo(uint8_t* dst, int row, const float (
     for (int q = 0; q < 4; ++q) {
       const float a = x[8 * c + 2 * q], b = x[8 * c + 2 * q + 1];
       const float ha = __bfloat162float(__float2bfloat16_rn(a)), hb = __bfloat162float(__float2bfloat16_rn(b));
-      hi[q] = pack2(ha, hb);
-      lo[q] = pack2(a - ha, b - hb);
+      hi[q] = ptx::pack_bf16(ha, hb);
+      lo[q] = ptx::pack_bf16(a - ha, b - hb);
     }
-    *reinterpret_cast<uint4*>(dst + swz128(row, c)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-    *reinterpret_cast<uint4*>(dst + kBox + swz128(row, c)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+    *reinterpret_cast<uint4*>(dst + ptx::swz128(row, c)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+    *reinterpret_cast<uint4*>(dst + kBox + ptx::swz128(row, c)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
   }
 }
 
@@ -246,12 +234,12 @@ flash_factored_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_cons
     for (int j = 8; j < kPos; ++j) mx[j & 7] = fmaxf(mx[j & 7], s[j]);
     const float m_new = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
                               fmaxf(fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])), m_run));
-    const float alpha = ex2(m_run - m_new);         // 0 on the first tile (m_run = -inf)
+    const float alpha = ptx::fast_exp2(m_run - m_new);         // 0 on the first tile (m_run = -inf)
 #pragma unroll
     for (int q = 0; q < 8; ++q) sm8[q] = 0.f;
 #pragma unroll
     for (int j = 0; j < kPos; ++j) {
-      s[j] = ex2(s[j] - m_new);                     // masked positions: 2^-inf = 0
+      s[j] = ptx::fast_exp2(s[j] - m_new);                     // masked positions: 2^-inf = 0
       sm8[j & 7] += s[j];
     }
     const float sum = ((sm8[0] + sm8[1]) + (sm8[2] + sm8[3])) + ((sm8[4] + sm8[5]) + (sm8[6] + sm8[7]));
@@ -259,9 +247,9 @@ flash_factored_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_cons
     m_run = m_new;
 #pragma unroll
     for (int c = 0; c < kPos / 8; ++c) {            // P as bf16, K-major: two boxes of 64 positions
-      const uint4 w = make_uint4(pack2(s[8 * c], s[8 * c + 1]), pack2(s[8 * c + 2], s[8 * c + 3]),
-                                 pack2(s[8 * c + 4], s[8 * c + 5]), pack2(s[8 * c + 6], s[8 * c + 7]));
-      *reinterpret_cast<uint4*>(sP + (c / 8) * kBox + swz128(tid, c % 8)) = w;
+      const uint4 w = make_uint4(ptx::pack_bf16(s[8 * c], s[8 * c + 1]), ptx::pack_bf16(s[8 * c + 2], s[8 * c + 3]),
+                                 ptx::pack_bf16(s[8 * c + 4], s[8 * c + 5]), ptx::pack_bf16(s[8 * c + 6], s[8 * c + 7]));
+      *reinterpret_cast<uint4*>(sP + (c / 8) * kBox + ptx::swz128(tid, c % 8)) = w;
     }
     ptx::fence_proxy_async_smem();
     ptx::tc_fence_before_sync();
@@ -340,11 +328,11 @@ flash_factored_kernel(const __grid_constant__ CUtensorMap tmC, const __grid_cons
     uint8_t* box = sC + (c0 / 64) * kBox;
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
-      const uint4 w = make_uint4(pack2(__uint_as_float(v[8 * c + 0]), __uint_as_float(v[8 * c + 1])),
-                                 pack2(__uint_as_float(v[8 * c + 2]), __uint_as_float(v[8 * c + 3])),
-                                 pack2(__uint_as_float(v[8 * c + 4]), __uint_as_float(v[8 * c + 5])),
-                                 pack2(__uint_as_float(v[8 * c + 6]), __uint_as_float(v[8 * c + 7])));
-      *reinterpret_cast<uint4*>(box + swz128(tid, (c0 % 64) / 8 + c)) = w;
+      const uint4 w = make_uint4(ptx::pack_bf16(__uint_as_float(v[8 * c + 0]), __uint_as_float(v[8 * c + 1])),
+                                 ptx::pack_bf16(__uint_as_float(v[8 * c + 2]), __uint_as_float(v[8 * c + 3])),
+                                 ptx::pack_bf16(__uint_as_float(v[8 * c + 4]), __uint_as_float(v[8 * c + 5])),
+                                 ptx::pack_bf16(__uint_as_float(v[8 * c + 6]), __uint_as_float(v[8 * c + 7])));
+      *reinterpret_cast<uint4*>(box + ptx::swz128(tid, (c0 % 64) / 8 + c)) = w;
     }
   }
   ptx::fence_proxy_async_smem();

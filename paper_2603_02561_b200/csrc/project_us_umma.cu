@@ -34,15 +34,6 @@ template <int D> struct UsCfg {
 };
 
 // byte offset of 16-byte chunk c of row `row` in a [rows][128 B] tile with the 128-byte swizzle
-__device__ __forceinline__ uint32_t swz(int row, int c) {
-  return (uint32_t)row * 128u + (uint32_t)((c ^ (row & 7)) << 4);
-}
-
-__device__ __forceinline__ uint32_t pack2(float a, float b) {
-  return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(a)) |
-         ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(b)) << 16);
-}
-
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 project_us_umma_kernel(const __grid_constant__ CUtensorMap tmap, const float* __restrict__ V,
@@ -102,7 +93,7 @@ project_us_umma_kernel(const __grid_constant__ CUtensorMap tmap, const float* __
     const float v = i < r ? V[((size_t)b * D + k) * r + i] : 0.f;
     const __nv_bfloat16 hi = __float2bfloat16_rn(v);
     const __nv_bfloat16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
-    const uint32_t off = (uint32_t)(k / 64) * v_tile + swz(i, (k % 64) / 8) + (k % 8) * 2;
+    const uint32_t off = (uint32_t)(k / 64) * v_tile + ptx::swz128(i, (k % 64) / 8) + (k % 8) * 2;
     *reinterpret_cast<__nv_bfloat16*>(sV + off) = hi;
     *reinterpret_cast<__nv_bfloat16*>(sV + Cfg::KB * v_tile + off) = lo;
   }
@@ -174,10 +165,10 @@ project_us_umma_kernel(const __grid_constant__ CUtensorMap tmap, const float* __
 #pragma unroll
             for (int c = 0; c < 4; ++c)
               if (c0 + 8 * c < r)
-                o4[c] = make_uint4(pack2(__uint_as_float(v[8 * c]), __uint_as_float(v[8 * c + 1])),
-                                   pack2(__uint_as_float(v[8 * c + 2]), __uint_as_float(v[8 * c + 3])),
-                                   pack2(__uint_as_float(v[8 * c + 4]), __uint_as_float(v[8 * c + 5])),
-                                   pack2(__uint_as_float(v[8 * c + 6]), __uint_as_float(v[8 * c + 7])));
+                o4[c] = make_uint4(ptx::pack_bf16(__uint_as_float(v[8 * c]), __uint_as_float(v[8 * c + 1])),
+                                   ptx::pack_bf16(__uint_as_float(v[8 * c + 2]), __uint_as_float(v[8 * c + 3])),
+                                   ptx::pack_bf16(__uint_as_float(v[8 * c + 4]), __uint_as_float(v[8 * c + 5])),
+                                   ptx::pack_bf16(__uint_as_float(v[8 * c + 6]), __uint_as_float(v[8 * c + 7])));
           } else {
 #pragma unroll
             for (int i = 0; i < 32; ++i)

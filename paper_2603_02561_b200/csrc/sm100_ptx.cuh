@@ -4,6 +4,7 @@
 #pragma once
 
 #include <cuda.h>
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -179,6 +180,28 @@ __device__ __forceinline__ void umma_bf16_ss(uint32_t tmem_d, uint64_t adesc, ui
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
+}
+
+// ---- small helpers of the tensor-core kernels ------------------------------------------------
+// Byte offset of 16-byte chunk c of row `row` in a 128-byte-swizzled tile of 128-byte rows.
+__device__ __forceinline__ uint32_t swz128(int row, int c) {
+  return (uint32_t)row * 128u + (uint32_t)((c ^ (row & 7)) << 4);
+}
+// The same for a 64-byte-swizzled tile of 64-byte rows (4 chunks per row; address bits 4-5 are
+// XORed with bits 7-8, i.e. with row / 2).
+__device__ __forceinline__ uint32_t swz64(int row, int c) {
+  return (uint32_t)row * 64u + (uint32_t)((c ^ ((row >> 1) & 3)) << 4);
+}
+// Two fp32 values rounded to bf16 (nearest even), `lo` in the low half of the word.
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+// 2^x by the special-function unit (2 ulp).
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 
 }  // namespace ptx
