@@ -601,7 +601,8 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
         "attn_apply": {"bound": "hbm", "achieved": ab["attn"] / (stage_ms["attn_apply"] * 1e-3) / 1e9,
                        "peak": pk["hbm_gbs"], "unit": "GB/s"},
         "eig": {"bound": "alu", "achieved": eflops / (stage_ms["eig"] * 1e-3) / 1e12, "peak": FP32_ALU_TFLOPS,
-                "unit": "TFLOP/s", "note": "serial Jacobi rounds on B of 148 SMs: latency-bound"},
+                "unit": "TFLOP/s", "note": "one CTA per user on B of 148 SMs, a chain of dependent steps (Householder reflections, Sturm counts, "
+                        "orthogonalisation, or Jacobi rounds in the fallback): latency-bound"},
         "attn_prepare": {"bound": "alu", "achieved": 6.0 * w.B * w.r * w.d * w.d / (stage_ms["attn_prepare"] * 1e-3) / 1e12,
                          "peak": FP32_ALU_TFLOPS, "unit": "TFLOP/s"},
     }

@@ -1034,7 +1034,8 @@ __device__ __forceinline__ void prepare_epilogue(float* __restrict__ sm, int b, 
   if (!vs_ready)
     for (int e = tid; e < D * rp; e += NT) {
       const int k = e / rp, i = e % rp;
-      VS[e] = i < r ? V[((size_t)b * D + k) * r + i] * S[(size_t)b * r + i] : 0.f;
+      // written earlier by this CTA: read through the L2, not the non-coherent path
+      VS[e] = i < r ? __ldcg(V + ((size_t)b * D + k) * r + i) * __ldcg(S + (size_t)b * r + i) : 0.f;
     }
   // Zero padding of the packed operands, 16 bytes at a time.  The tensor-core attention kernel
   // multiplies over np = 16 ceil(r / 16) token slots only (slots r .. r8-1, r8 = r rounded up to
