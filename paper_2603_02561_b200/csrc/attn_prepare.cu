@@ -11,6 +11,7 @@
 // Two CTAs per user: one computes Key_r^T and T (W_K, W_Q), the other Value_r (W_V).
 // Each weight matrix is staged once in shared memory with coalesced 16-byte loads; the small
 // products then run out of shared memory with 4 outputs per thread.
+#include "project_mma.cuh"
 #include "solar_internal.cuh"
 
 namespace solar {
@@ -141,6 +142,43 @@ attn_prepare_kernel(const float* __restrict__ S, const float* __restrict__ V,
   }
 }
 
+// bf16 weights, d = 64 or 128: one CTA per user, the three products on the tensor cores (the
+// routine the eigensolver's epilogue uses, so a forward pass gives the same bits either way).
+template <int D>
+__global__ void __launch_bounds__(D == 128 ? 256 : 128, 1)
+attn_prepare_mma_kernel(const float* __restrict__ S, const float* __restrict__ V, const void* __restrict__ Wq,
+                        const void* __restrict__ Wk, const void* __restrict__ Wv, float scale, int r,
+                        char* __restrict__ ws, AttnWs lay) {
+  constexpr int NT = D == 128 ? 256 : 128;
+  extern __shared__ __align__(16) unsigned char smb[];
+  const int rp = (r + 3) & ~3;
+  const int b = blockIdx.x, tid = threadIdx.x;
+  char* wsb = ws + (size_t)b * lay.per_user;
+  float* VS = reinterpret_cast<float*>(smb);     // [D][rp]  V Sigma (zero in the padding)
+  pdl_wait();                                    // as in the kernel above
+  for (int e = tid; e < D * rp; e += NT) {
+    const int k = e / rp, i = e % rp;
+    VS[e] = i < r ? V[((size_t)b * D + k) * r + i] * (S != nullptr ? S[(size_t)b * r + i] : 1.f) : 0.f;
+  }
+  __syncthreads();
+  pdl_trigger();
+  pmma::project<D, NT>(smb, r, Wq, Wk, Wv, scale, reinterpret_cast<__nv_bfloat16*>(wsb + lay.tpk_off),
+                       reinterpret_cast<__nv_bfloat16*>(wsb + lay.vpk_off), reinterpret_cast<float*>(wsb + lay.tf_off),
+                       reinterpret_cast<float*>(wsb + lay.vr_off), kTokenSlots, tid);
+}
+
+template <int D>
+cudaError_t launch_mma(int B, int r, const float* S, const float* V, const void* Wq, const void* Wk, const void* Wv,
+                       float scale, char* ws, const AttnWs& lay, cudaStream_t st) {
+  static bool limits_set[kMaxDevicesCached] = {};
+  cudaError_t e = set_kernel_limits(reinterpret_cast<const void*>(&attn_prepare_mma_kernel<D>),
+                                    (size_t)pmma::Lay<D>::bytes(kTokenSlots), limits_set);
+  if (e != cudaSuccess) return e;
+  e = launch_pdl(attn_prepare_mma_kernel<D>, dim3(B), dim3(D == 128 ? 256 : 128),
+                 (size_t)pmma::Lay<D>::bytes((r + 15) & ~15), st, S, V, Wq, Wk, Wv, scale, r, ws, lay);
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
 template <typename T>
 cudaError_t launch_t(int B, int d, int r, const float* S, const float* V, const void* Wq,
                      const void* Wk, const void* Wv, float scale, char* ws, const AttnWs& lay,
@@ -175,6 +213,8 @@ cudaError_t launch_t(int B, int d, int r, const float* S, const float* V, const 
 cudaError_t launch_attn_prepare(int B, int d, int r, solar_dtype_t dt, const float* S,
                                 const float* V, const void* Wq, const void* Wk, const void* Wv,
                                 float scale, char* ws, const AttnWs& lay, cudaStream_t st) {
+  if (dt == SOLAR_BF16 && d == 64) return launch_mma<64>(B, r, S, V, Wq, Wk, Wv, scale, ws, lay, st);
+  if (dt == SOLAR_BF16 && d == 128) return launch_mma<128>(B, r, S, V, Wq, Wk, Wv, scale, ws, lay, st);
   return dt == SOLAR_BF16
              ? launch_t<__nv_bfloat16>(B, d, r, S, V, Wq, Wk, Wv, scale, ws, lay, st)
              : launch_t<float>(B, d, r, S, V, Wq, Wk, Wv, scale, ws, lay, st);

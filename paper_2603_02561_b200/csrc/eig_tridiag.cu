@@ -37,6 +37,7 @@
 // Householder loop is cut into stages with fixed live rows and columns), keeps divisions off
 // the dependency chains, and spreads independent work over the warps.
 #include "eig_jacobi.cuh"
+#include "project_mma.cuh"
 
 namespace solar {
 
@@ -78,7 +79,10 @@ template <int D, int RP> struct TriSmem {
   static constexpr int KT = SG + RP;                             // [RP] twist index (int)
   static constexpr int PART = KT + RP;                           // [2][NW][RP] per-warp partial results
   static constexpr int TRI_FLOATS = PART + 2 * C::NW * RP;
-  static constexpr int EPI_FLOATS = 2 * D * RP + 2 * D * D;      // the projection epilogue: V Sigma, Key_r^T, two weights
+  // the projection epilogue: V Sigma, Key_r^T, two weights (FFMA form) or the tensor-core form's staging
+  static constexpr int EPI_FFMA = 2 * D * RP + 2 * D * D;
+  static constexpr int EPI_MMA = (D >= 64) ? pmma::Lay<(D >= 64 ? D : 64)>::bytes(RP) / 4 : 0;
+  static constexpr int EPI_FLOATS = EPI_FFMA > EPI_MMA ? EPI_FFMA : EPI_MMA;
   static constexpr int M1 = TRI_FLOATS > full_jacobi_floats<D>() ? TRI_FLOATS : full_jacobi_floats<D>();
   static constexpr int FLOATS = M1 > EPI_FLOATS ? M1 : EPI_FLOATS;
   static constexpr size_t BYTES = (size_t)FLOATS * sizeof(float);
@@ -1029,6 +1033,19 @@ __device__ __forceinline__ void prepare_epilogue(float* __restrict__ sm, int b, 
   constexpr int MAXT = 2;               // tiles per thread (kept in registers across a barrier)
   const uint4 z4 = make_uint4(0u, 0u, 0u, 0u);
 
+  if (D >= 64 && fa.mode == 1 && !fa.write_f32) {
+    // bf16 weights: the three products on the tensor cores
+    if (!vs_ready) {
+      for (int e = tid; e < D * rp; e += NT) {
+        const int k = e / rp, i = e % rp;
+        VS[e] = i < r ? __ldcg(V + ((size_t)b * D + k) * r + i) * __ldcg(S + (size_t)b * r + i) : 0.f;
+      }
+      __syncthreads();
+    }
+    pmma::project<(D >= 64 ? D : 64), NT>(reinterpret_cast<unsigned char*>(sm), r, fa.Wq, fa.Wk, fa.Wv, fa.scale, Tpk, Vpk,
+                                          nullptr, nullptr, (r + 15) & ~15, tid);
+    return;
+  }
   stage_weight_any<D, NT, false>(fa.Wk, fa.mode, W0, tid);
   stage_weight_any<D, NT, true>(fa.Wq, fa.mode, W1, tid);
   if (!vs_ready)
