@@ -12,7 +12,8 @@ The timed region replays CUDA graphs of whole steps (no host work between kernel
 --in-flight S > 1, S independent batches are in flight on S streams (each with its own
 workspace and factors), which is how a serving process overlaps one request's eigensolve
 (B CTAs) with another's streaming passes; S = 1 gives the single-call latency.  Both
-figures are printed; `value` is the one at the S given (default 24).  Every step in flight
+figures are printed; `value` is the one at the S given (default 30: the step time falls up
+to 31 streams and jumps by a fifth at 32, where streams start to share a hardware queue).  Every step in flight
 reads and writes buffers of its own (2 S + 7 buffer sets), --steps is a minimum, and the
 timed region lasts at least half a second; the spread over the graph replays is printed.
 `value` is measured through solar_svd_attention_fused (three launches per step); the same
@@ -241,7 +242,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3")
-    ap.add_argument("--in-flight", type=int, default=24, help="independent batches in flight (streams)")
+    ap.add_argument("--in-flight", type=int, default=30, help="independent batches in flight (streams)")
     ap.add_argument("--path", default="fused", choices=["fused", "two_call"],
                     help="which public call `value` is measured through (the other is printed beside it)")
     ap.add_argument("--cpu-users", type=int, default=8, help="users in the cpu_baseline sample")
