@@ -242,6 +242,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3")
+    ap.add_argument("--rounds", type=int, default=24,
+                    help="consecutive steps of a lane in one CUDA graph (the lanes drain and refill between replays)")
     ap.add_argument("--in-flight", type=int, default=30, help="independent batches in flight (streams)")
     ap.add_argument("--path", default="fused", choices=["fused", "two_call"],
                     help="which public call `value` is measured through (the other is printed beside it)")
@@ -390,7 +392,7 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
             step(0, lane, main_stream, path)
     torch.cuda.synchronize()
 
-    ROUNDS = 12
+    ROUNDS = max(1, args.rounds)
     other = "two_call" if args.path == "fused" else "fused"
     g_main = capture(ROUNDS, lanes)
     g_other = capture(ROUNDS, lanes, other) if not light else None
