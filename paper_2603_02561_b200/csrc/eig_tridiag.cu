@@ -217,12 +217,15 @@ __device__ __forceinline__ void tri_stage(float (&a)[TriCfg<D>::RPT][TriCfg<D>::
     for (int w = 0; w < NW; ++w) { pvs += pvp[par * 8 + w]; pk1 += tpart[(par * NW + w) * D + k1]; }
     const float kk = 0.5f * beta * beta * pvs;
     const float wk1 = fmaf(-kk, vk1, beta * pk1);
-    float wr[RPT], wc[NG][4];
+    float wr[RPT], wc[NG][4], prow[RPT];
+#pragma unroll
+    for (int q = 0; q < RPT; ++q) prow[q] = 0.f;
 #pragma unroll
     for (int q = Q0; q < RPT; ++q) {
       float t = 0.f;
 #pragma unroll
       for (int w = 0; w < NW; ++w) t += tpart[(par * NW + w) * D + lane + 32 * q];
+      prow[q] = t;
       wr[q] = (lane + 32 * q > k) ? fmaf(-kk, vr[q], beta * t) : 0.f;
       // column k+1 of the updated matrix at my rows: row k+1 before the update, corrected
       xr[q] = fmaf(-wr[q], vk1, fmaf(-vr[q], wk1, xpre[par * D + lane + 32 * q]));
@@ -230,14 +233,13 @@ __device__ __forceinline__ void tri_stage(float (&a)[TriCfg<D>::RPT][TriCfg<D>::
 #pragma unroll
     for (int g = G0; g < NG; ++g) {
       const int cb = 4 * (warp + NW * g);
-      float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-      for (int w = 0; w < NW; ++w) {
-        const float4 u = *reinterpret_cast<const float4*>(tpart + (par * NW + w) * D + cb);
-        t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
-      }
       const float4 xp = *reinterpret_cast<const float4*>(xpre + par * D + cb);
-      const float tt[4] = {t.x, t.y, t.z, t.w}, xx[4] = {xp.x, xp.y, xp.z, xp.w};
+      const float xx[4] = {xp.x, xp.y, xp.z, xp.w};
+      float tt[4];
+      // (A v) at column cb + c is the row sum held by the lane that owns row cb + c (slot
+      // 4 NW g / 32 of that lane): one shuffle instead of NW loads and adds
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tt[c] = __shfl_sync(kFull, prow[(4 * NW * g) >> 5], (cb + c) & 31);
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         wc[g][c] = (cb + c > k) ? fmaf(-kk, vc[g][c], beta * tt[c]) : 0.f;
