@@ -801,6 +801,10 @@ __device__ __forceinline__ bool eig_user(const float* __restrict__ gpart, const 
       }
       __syncthreads();
       float* t = Vc; Vc = Vn; Vn = t;
+      // With E = L + diag + L^T the pass leaves (I - L)(I + E)(I - L^T) = I + diag - L L^T - L^2 -
+      // (L^T)^2 + O(E^3), and the scaling removes the diagonal: what remains off the diagonal is
+      // below 3 r max|E|^2.  Where that is a quarter of the bound, V^T V is not formed again.
+      if (3.f * (float)r * em * em <= 0.25f * tol.ortho) break;
     }
     __syncthreads();      // G is staged; E and the vectors are settled
 
