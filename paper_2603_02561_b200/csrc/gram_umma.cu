@@ -28,9 +28,12 @@ template <int D> struct GramCfg {
   static constexpr int BOXES = D / 64;                       // 64-column TMA boxes per tile
   static constexpr int BOX_BYTES = kTileRows * 128;          // 16 KB: 128 rows x 64 bf16
   static constexpr int TILE_BYTES = BOXES * BOX_BYTES;
-  // Four 16/32 KB stages keep more than one SM's share of the HBM latency-bandwidth product in
-  // flight and leave room for two eigensolver CTAs (78 KB each at d = 64) beside a Gram CTA.
-  static constexpr int STAGES = 4;
+  // Three 16 KB stages at d = 64 (four of 32 KB at d = 128).  Alone a deeper ring changes nothing
+  // (7.9 us either way); with many requests in flight the CTA's shared-memory footprint is what
+  // counts -- the step takes 8.87 / 8.63 / 8.49 / 8.67 us with 5 / 4 / 3 / 2 stages on the
+  // 16 x 10240 x 64 serving shape -- because the Gram, eigensolver and attention CTAs of different
+  // requests share every SM's 227 KB.
+  static constexpr int STAGES = (D == 64) ? 3 : 4;
   static constexpr size_t SMEM = (size_t)STAGES * TILE_BYTES + 1024;   // + slack to align to 1024
   static constexpr uint32_t IDESC = ptx::umma_idesc_bf16(D, D, true, true);
 };
