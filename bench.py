@@ -16,6 +16,9 @@ figures are printed; `value` is the one at the S given (default 30: the step tim
 to 31 streams and jumps by a fifth at 32, where streams start to share a hardware queue).  Every step in flight
 reads and writes buffers of its own (2 S + 7 buffer sets), --steps is a minimum, and the
 timed region lasts at least half a second; the spread over the graph replays is printed.
+The steps in flight run under solar_set_slice_limit(--slice-limit, default 2: few long slices
+per user, the setting for throughput); `single_call` is taken under the library's default
+slicing (the setting for latency), the other combination of each is printed beside it.
 `value` is measured through solar_svd_attention_fused (three launches per step); the same
 measurement through solar_lowrank_factor + solar_svd_attention_fwd (four launches) is
 printed beside it as `two_call`.
@@ -242,6 +245,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c3")
+    ap.add_argument("--slice-limit", type=int, default=2,
+                    help="solar_set_slice_limit for the steps in flight (0 = the library's own slicing, chosen for the "
+                         "latency of one call); the single-call figure is always taken with 0")
     ap.add_argument("--rounds", type=int, default=24,
                     help="consecutive steps of a lane in one CUDA graph (the lanes drain and refill between replays)")
     ap.add_argument("--in-flight", type=int, default=30, help="independent batches in flight (streams)")
@@ -394,8 +400,19 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
 
     ROUNDS = max(1, args.rounds)
     other = "two_call" if args.path == "fused" else "fused"
+    # The slicing of the streaming passes is baked into a graph when it is captured.  Requests in
+    # flight run under the throughput setting (few, long slices); one call at a time under the
+    # library's default (slices that fill the GPU once).  Workspaces were sized under the default,
+    # which is the larger.
+    slice_cap = max(0, args.slice_limit) if n_lanes > 1 else 0
+    solar.set_slice_limit(slice_cap)
+    slices_in_flight = solar.gram_slices(w.B, w.N, w.d, tdt)
     g_main = capture(ROUNDS, lanes)
     g_other = capture(ROUNDS, lanes, other) if not light else None
+    g_single_cap = capture(nb, lanes[:1]) if (n_lanes > 1 and slice_cap > 0) else None
+    solar.set_slice_limit(0)
+    slices_default = solar.gram_slices(w.B, w.N, w.d, tdt)
+    g_main_default = capture(ROUNDS, lanes) if (slice_cap > 0 and not light) else None
     g_single = capture(nb, lanes[:1]) if n_lanes > 1 else g_main
     # warm-up (at least 3 steps and the --warmup asked for), which also calibrates the plan
     warm = max(1, -(-max(args.warmup, 3) // (ROUNDS * n_lanes)))
@@ -432,6 +449,20 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
     sev = timed_replays(g_single, single_reps)
     sync_all()
     ms_single = sev[0].elapsed_time(sev[-1]) / (single_reps * (nb if n_lanes > 1 else steps_per_graph))
+    ms_single_cap = None
+    if g_single_cap is not None:
+        g_single_cap.replay()
+        sevc = timed_replays(g_single_cap, single_reps)
+        sync_all()
+        ms_single_cap = sevc[0].elapsed_time(sevc[-1]) / (single_reps * nb)
+    default_plan = None
+    if g_main_default is not None:
+        g_main_default.replay()
+        evd = timed_replays(g_main_default, max(10, replays // 4))
+        sync_all()
+        default_plan = {"ms_per_step": evd[0].elapsed_time(evd[-1]) / ((len(evd) - 1) * steps_per_graph),
+                        "spread": bp.spread(per_replay_ms(evd), steps_per_graph), "gram_slices": slices_default,
+                        "what": "the same steps in flight under the library's default slicing (slice limit 0)"}
     # ... and as plain calls (no graph): what a caller without graphs pays per step, host work included
     plain_n = 50
     for _ in range(5):
@@ -623,13 +654,17 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
                    "storage": w.dtype, "users_per_gpu": w.B, "in_flight": n_lanes, "path": args.path,
                    "launch": f"CUDA graphs of {steps_per_graph} steps ({ROUNDS} per lane), {replays} replays, "
                              f"{ms * 1e-3:.2f} s timed",
+                   "slice_limit": slice_cap, "gram_slices": slices_in_flight,
                    "distinct_batches": nb, "seeded_batches": nseed,
                    "l2": f"every step in flight has its own input and output buffers: {nb} buffer sets "
                          f"({nb * ab['total'] / 2**20:.0f} MiB > 126 MiB L2), {nseed} seeded batches and device "
                          "copies of them with the users rotated"},
         "ms_per_step_spread": spread_main,
         "single_call": {"ms_per_step": ms_single, "value": world * w.pairs / (ms_single * 1e-3),
-                        "note": "one step at a time on one stream (in_flight = 1), graph replay",
+                        "note": "one step at a time on one stream (in_flight = 1), graph replay, the library's "
+                                "default slicing (slice limit 0)",
+                        "gram_slices": slices_default,
+                        "ms_per_step_with_slice_limit": ms_single_cap,
                         "plain_calls_ms_per_step": ms_plain,
                         "plain_calls_note": "the same without a graph: host launch work included"},
         ("two_call" if args.path == "fused" else "fused"): (None if ms_other is None else {
@@ -637,6 +672,7 @@ def measure(args, w, torch, dist, solar, world, rank, local, light=False):
             "frac": (w.pairs / (ms_other * 1e-3)) / (w.pairs / roof_s),
             "what": ("solar_lowrank_factor + solar_svd_attention_fwd (four launches per step)"
                      if args.path == "fused" else "solar_svd_attention_fused (three launches per step)")}),
+        "default_slicing_in_flight": default_plan,
         "path_roofline": {"bound": "hbm", "algorithmic_bytes": ab["total"],
                           "algorithmic_flops": algorithmic_flops(w),
                           "roofline_pairs_per_s": w.pairs / roof_s, "frac": value / world / (w.pairs / roof_s),

@@ -166,6 +166,23 @@ solar_status_t solar_svd_attention_fused(int B, int M, int N, int d, int r, sola
  * checked on its own; argument meaning and rules are those given above.
  * ------------------------------------------------------------------------- */
 
+/* Tuning knob, process-wide: the largest number of row slices (CTAs) a user's history is cut
+ * into by the streaming passes over H (the Gram pass of Eq. 9's factorization, U Sigma = H V,
+ * dH = H K); 0, the default, means no cap.  Without a cap the slicing is chosen for the latency
+ * of ONE call: B * slices CTAs fill the GPU once (B = 16, N = 10240: nine slices).  A process
+ * that keeps many independent calls in flight on different streams is better served by fewer,
+ * longer slices (two or three): every CTA pays its fixed start-up and wind-down while holding
+ * shared memory that other requests' CTAs could use, and the eigensolver adds up fewer partial
+ * matrices -- measured on that shape with 30 requests in flight: 8.5 us per request at nine
+ * slices, 7.9 at three, 7.8 at two, for 66 / 71 / 77 us of latency per single call.
+ * Results agree to rounding (the partial sums are grouped differently), not bit for bit.
+ * Set it before sizing workspaces: the *_workspace_bytes functions follow the current value,
+ * and a call made under a higher cap than its workspace was sized for returns
+ * SOLAR_ERR_WORKSPACE.  Keep it unchanged between a stage call that writes a workspace
+ * (solar_gram_partials) and the stage calls that read it.  Returns the previous value.  Safe to
+ * call from any thread; calls already enqueued are not affected. */
+int solar_set_slice_limit(int max_slices);
+
 /* Number of partial Gram matrices solar_gram_partials leaves per user (>= 1), and
  * the number of row slices (CTAs, status words) per user behind them (a multiple of it). */
 int solar_gram_splits(int B, int N, int d, solar_dtype_t dt);

@@ -1,6 +1,15 @@
 // C ABI of the SVD-Attention forward pass: argument checks, workspace layout,
 // kernel selection.  Every host-visible error is returned before any launch.
+#include <atomic>
+
 #include "solar_internal.cuh"
+
+namespace solar {
+namespace {
+std::atomic<int> g_slice_limit{0};     // solar_set_slice_limit
+}  // namespace
+int slice_limit() { return g_slice_limit.load(std::memory_order_relaxed); }
+}  // namespace solar
 
 using namespace solar;
 
@@ -67,6 +76,11 @@ size_t solar_workspace_bytes(int B, int M, int N, int d, int r, solar_dtype_t dt
   const size_t f = factor_ws_bytes(B, N, d, dt), a = attn_ws_bytes(B, d, r);
   const size_t need = f > a ? f : a;
   return need ? need : 256;
+}
+
+int solar_set_slice_limit(int max_slices) {
+  if (max_slices < 0) max_slices = 0;
+  return solar::g_slice_limit.exchange(max_slices);
 }
 
 int solar_gram_splits(int B, int N, int d, solar_dtype_t dt) {

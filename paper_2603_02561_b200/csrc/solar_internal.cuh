@@ -37,11 +37,16 @@ inline long slice_cost(int B, int tiles, int s, int* s_eff_out, int* chunk_out) 
   return waves * (chunk + 2);
 }
 
+// Process-wide cap on the slices per user (solar_set_slice_limit; 0 = none).
+int slice_limit();
+
 inline GramPlan slice_plan(int B, int N) {
   GramPlan p;
   p.tiles = (N + kGramTileRows - 1) / kGramTileRows;
   long best_cost = -1;
-  const int smax = p.tiles < kMaxSplits ? p.tiles : kMaxSplits;
+  int smax = p.tiles < kMaxSplits ? p.tiles : kMaxSplits;
+  const int cap = slice_limit();
+  if (cap > 0 && cap < smax) smax = cap;
   p.splits = 1; p.chunk_tiles = p.tiles;
   for (int s = 1; s <= smax; ++s) {
     int s_eff, chunk;
@@ -66,7 +71,9 @@ inline GramPlan gram_plan(int B, int N, bool clustered) {
   GramPlan p;
   p.tiles = (N + kGramTileRows - 1) / kGramTileRows;
   long best_cost = -1;
-  const int smax = p.tiles < kMaxSplits ? p.tiles : kMaxSplits;
+  int smax = p.tiles < kMaxSplits ? p.tiles : kMaxSplits;
+  const int cap = slice_limit();
+  if (cap > 0 && cap < smax) smax = cap;
   p.splits = 1; p.chunk_tiles = p.tiles;
   for (int s = 1; s <= smax; ++s) {
     int s_eff, chunk;

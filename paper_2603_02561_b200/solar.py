@@ -38,6 +38,7 @@ SIGNATURES = {
     "solar_fused_workspace_bytes": (_c_size, [_c_int] * 5 + [_c_int]),
     "solar_svd_attention_fused": (_c_int, [_c_int] * 5 + [_c_int] + [_c_vp] * 5 + [_c_float, _c_uint] +
                                   [_c_vp] * 4 + [_c_vp, _c_size, _c_vp]),
+    "solar_set_slice_limit": (_c_int, [_c_int]),
     "solar_gram_splits": (_c_int, [_c_int] * 3 + [_c_int]),
     "solar_gram_slices": (_c_int, [_c_int] * 3 + [_c_int]),
     "solar_gram_partials": (_c_int, [_c_int] * 3 + [_c_int, _c_vp, _c_vp, _c_size, _c_vp]),
@@ -293,6 +294,11 @@ def attn_apply(C, r, flags, O, workspace, stream=None):
     _check(lib().solar_attn_apply(B, M, d, r, dtype_code(C.dtype), _ptr(C), int(flags), _ptr(O),
                                   _ptr(workspace), workspace.numel(), _stream(stream)),
            "solar_attn_apply")
+
+
+def set_slice_limit(max_slices: int) -> int:
+    """solar_set_slice_limit: process-wide cap on the row slices per user (0 = none); returns the old value."""
+    return int(lib().solar_set_slice_limit(int(max_slices)))
 
 
 def fused_workspace_bytes(B, M, N, d, r, dtype) -> int:

@@ -119,3 +119,23 @@ def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
     monkeypatch.setattr(solar, "LIB_PATH", str(tmp_path / "missing.so"))
     with pytest.raises(RuntimeError, match="no CPU fallback"):
         solar.lib()
+
+
+def test_slice_limit_is_a_host_side_setting():
+    """solar_set_slice_limit needs no GPU: it returns the previous value, caps the slice count
+    the planning calls report, and never makes a workspace larger."""
+    from paper_2603_02561_b200 import solar
+    L = solar.lib()
+    args = (16, 2048, 10240, 64, 32, solar.BF16)
+    old = L.solar_set_slice_limit(0)
+    try:
+        n0 = L.solar_gram_slices(16, 10240, 64, solar.BF16)
+        b0 = L.solar_workspace_bytes(*args)
+        assert n0 == 9
+        assert L.solar_set_slice_limit(3) == 0
+        assert L.solar_gram_slices(16, 10240, 64, solar.BF16) == 3
+        assert L.solar_workspace_bytes(*args) <= b0
+        assert L.solar_set_slice_limit(-5) == 3           # negative means no cap
+        assert L.solar_gram_slices(16, 10240, 64, solar.BF16) == n0
+    finally:
+        L.solar_set_slice_limit(old)

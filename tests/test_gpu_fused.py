@@ -112,3 +112,36 @@ def test_inputs_written_by_the_kernel_just_before_the_call(fused):
             torch.cuda.synchronize()
             assert torch.equal(S, ref[0]) and torch.equal(V, ref[1])
             assert torch.equal(O.view(torch.uint8), ref[2].view(torch.uint8))
+
+
+def test_slice_limit_changes_the_slicing_not_the_result():
+    """solar_set_slice_limit: fewer, longer row slices per user (the setting for throughput with many
+    requests in flight).  The partial sums are grouped differently, so the factors agree to rounding
+    and the output within the parity tolerance; the oracle is matched either way; a workspace sized
+    under a cap is refused once the cap is lifted."""
+    w = wl.CONFIGS["c3"].with_(B=3, N=5000, M=300)
+    inp = wl.generate(w)
+    H, C, Wq, Wk, Wv = _dev(w, inp)
+    old = solar.set_slice_limit(0)
+    try:
+        n_default = solar.gram_slices(w.B, w.N, w.d, H.dtype)
+        O0, S0, V0 = solar.svd_attention_fused(H, C, Wq, Wk, Wv, w.r, inp["scale"])
+        assert solar.set_slice_limit(2) == 0
+        assert solar.gram_slices(w.B, w.N, w.d, H.dtype) == 2 < n_default
+        small = solar.alloc_fused_workspace(w.B, w.M, w.N, w.d, w.r, H.dtype)
+        O2, S2, V2 = solar.svd_attention_fused(H, C, Wq, Wk, Wv, w.r, inp["scale"], workspace=small)
+        S2b, V2b = solar.lowrank_factor(H, w.r)                       # the two-call path follows the cap too
+        torch.cuda.synchronize()
+        assert torch.equal(S2, S2b) and torch.equal(V2, V2b)
+        assert (S2 - S0).abs().max() <= 1e-5 * S0.max()
+        got = {"S": S2.cpu().numpy().astype(np.float64), "V": V2.cpu().numpy().astype(np.float64),
+               "O": O2.float().cpu().numpy().astype(np.float64)}
+        for k in range(w.B):
+            assert ph.compare_user(w, inp, got, k)["o_err"] <= ph.TOL[w.dtype]
+        assert solar.set_slice_limit(0) == 2
+        assert small.numel() < solar.fused_workspace_bytes(w.B, w.M, w.N, w.d, w.r, H.dtype)
+        with pytest.raises(solar.SolarError) as e:
+            solar.svd_attention_fused(H, C, Wq, Wk, Wv, w.r, inp["scale"], workspace=small)
+        assert e.value.status == solar.ERR_WORKSPACE
+    finally:
+        solar.set_slice_limit(old)
