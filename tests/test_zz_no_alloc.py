@@ -8,6 +8,8 @@ Collected last on purpose: a run that stops at the first failure has then alread
 other test."""
 import ctypes
 
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -66,10 +68,16 @@ def test_static_scratch_variant_allocates_nothing():
     info = torch.empty(w.B, dtype=torch.int32, device="cuda")
     solar.lowrank_factor_static(H, w.r, S=S, V=V, info=info)          # first call: set-up
     torch.cuda.synchronize()
-    before = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), torch.cuda.mem_get_info()[0])
-    for _ in range(3):
-        solar.lowrank_factor_static(H, w.r, S=S, V=V, info=info)
-    torch.cuda.synchronize()
-    after = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), torch.cuda.mem_get_info()[0])
+    # tensors left behind by earlier tests must not be freed inside the measured window
+    gc.collect()
+    gc.disable()
+    try:
+        before = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), torch.cuda.mem_get_info()[0])
+        for _ in range(3):
+            solar.lowrank_factor_static(H, w.r, S=S, V=V, info=info)
+        torch.cuda.synchronize()
+        after = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), torch.cuda.mem_get_info()[0])
+    finally:
+        gc.enable()
     assert before == after, (before, after)
     assert (info == 0).all()
