@@ -368,8 +368,9 @@ cudaError_t launch_dr(int B, int M, int N, const void* C, const void* US, void* 
   ok = ok && encode_tmap_bf16_3d_sw(&tmUS, US, R, (uint64_t)N, (uint64_t)B, (uint64_t)R * 2, (uint64_t)N * R * 2, R,
                                     kPos, Cfg::RB);
   if (!ok) return cudaErrorInvalidValue;
-  cudaError_t e = cudaFuncSetAttribute(flash_factored_kernel<D, R>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)Cfg::SMEM);
+  static bool limits_set[kMaxDevicesCached] = {};
+  const cudaError_t e = set_kernel_limits(reinterpret_cast<const void*>(&flash_factored_kernel<D, R>), Cfg::SMEM,
+                                          limits_set);
   if (e != cudaSuccess) return e;
   const dim3 grid((M + kRows - 1) / kRows, B), block(128);
   return launch_pdl(flash_factored_kernel<D, R>, grid, block, Cfg::SMEM, st, tmC, tmO, tmT, tmV, tmUS, N, M,
