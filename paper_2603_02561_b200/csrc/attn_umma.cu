@@ -271,6 +271,8 @@ bool attn_umma_supported(int d, solar_dtype_t dt) { return dt == SOLAR_BF16 && (
 
 cudaError_t launch_attn_umma(int B, int M, int d, int r, const void* C, unsigned flags, void* O,
                              const char* ws, const AttnWs& lay, bool early_c, cudaStream_t st) {
+  if (slice_limit() > 0 && attn_pipe_supported(M, d, r, SOLAR_BF16))
+    return launch_attn_pipe(B, M, r, C, flags, O, ws, lay, early_c, st);
   return d == 64 ? launch_d<64>(B, M, r, C, flags, O, ws, lay, early_c, st)
                  : launch_d<128>(B, M, r, C, flags, O, ws, lay, early_c, st);
 }

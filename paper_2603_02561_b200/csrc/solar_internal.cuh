@@ -234,6 +234,11 @@ bool flash_factored_supported(int d, int r, solar_dtype_t dt);
 cudaError_t launch_flash_factored(int B, int M, int N, int d, int r, const void* C, const void* US, void* O,
                                   const char* ws, const AttnWs& lay, cudaStream_t st);
 bool attn_umma_supported(int d, solar_dtype_t dt);
+// Throughput form of the tensor-core attention kernel: long CTAs that overlap the candidate
+// stream, the GEMMs and the softmax of consecutive tiles (chosen under a slice limit).
+bool attn_pipe_supported(int M, int d, int r, solar_dtype_t dt);
+cudaError_t launch_attn_pipe(int B, int M, int r, const void* C, unsigned flags, void* O, const char* ws,
+                             const AttnWs& lay, bool early_c, cudaStream_t st);
 cudaError_t launch_attn_umma(int B, int M, int d, int r, const void* C, unsigned flags, void* O,
                              const char* ws, const AttnWs& lay, bool early_c, cudaStream_t st);
 

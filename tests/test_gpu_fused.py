@@ -145,3 +145,33 @@ def test_slice_limit_changes_the_slicing_not_the_result():
         assert e.value.status == solar.ERR_WORKSPACE
     finally:
         solar.set_slice_limit(old)
+
+
+@pytest.mark.parametrize("M,r,flags", [(2048, 32, 0), (1000, 27, 0), (3000, 16, 0), (515, 5, 0),
+                                       (1300, 32, solar.FLAG_NO_SOFTMAX)])
+def test_throughput_attention_kernel_gives_the_same_bits(M, r, flags):
+    """Under a slice limit the candidate attention runs as long CTAs that overlap the candidate
+    stream, the GEMMs and the softmax of consecutive tiles (bf16, d = 64, r <= 32, at least four
+    tiles).  Same GEMMs in the same order, same softmax: the output must equal the
+    one-tile-per-CTA kernel's bit for bit, ragged last tile included."""
+    w = wl.CONFIGS["c3"].with_(B=3, N=1500, M=M, r=r)
+    inp = wl.generate(w)
+    H, C, Wq, Wk, Wv = _dev(w, inp)
+    old = solar.set_slice_limit(0)
+    try:
+        ws = solar.alloc_workspace(w.B, w.M, w.N, w.d, w.r, H.dtype)
+        S, V = solar.lowrank_factor(H, w.r, workspace=ws, M=w.M)
+        O0 = torch.full_like(C, float("nan"))
+        solar.svd_attention_fwd(C, S, V, Wq, Wk, Wv, inp["scale"], flags, O=O0, workspace=ws, N=w.N)
+        solar.set_slice_limit(2)
+        guard = torch.full((w.B, w.M + 128, w.d), 7.0, dtype=C.dtype, device="cuda")    # rows past M stay untouched
+        O1 = guard[:, :w.M]
+        O1c = torch.full_like(C, float("nan"))
+        for _ in range(2):
+            solar.svd_attention_fwd(C, S, V, Wq, Wk, Wv, inp["scale"], flags, O=O1c, workspace=ws, N=w.N)
+        torch.cuda.synchronize()
+        assert torch.equal(O1c.view(torch.uint8), O0.view(torch.uint8))
+        assert not torch.isnan(O1c.float()).any()
+        del O1, guard
+    finally:
+        solar.set_slice_limit(old)
