@@ -175,6 +175,11 @@ solar_status_t solar_svd_attention_fused(int B, int M, int N, int d, int r, sola
  * shared memory that other requests' CTAs could use, and the eigensolver adds up fewer partial
  * matrices -- measured on that shape with 30 requests in flight: 8.5 us per request at nine
  * slices, 7.9 at three, 7.8 at two, for 66 / 71 / 77 us of latency per single call.
+ * A positive value is read as "this process wants throughput" by the other kernels too: the
+ * candidate attention (bf16, d = 64, r <= 32, M >= 512) then runs as a few long CTAs per user
+ * that overlap the candidate stream, the GEMMs and the softmax of consecutive tiles -- the same
+ * bits in O -- and the eigensolver releases it a little later; together 7.6 us per request in
+ * flight and about 100 us for a lone call.
  * Results agree to rounding (the partial sums are grouped differently), not bit for bit.
  * Set it before sizing workspaces: the *_workspace_bytes functions follow the current value,
  * and a call made under a higher cap than its workspace was sized for returns
